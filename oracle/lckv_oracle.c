@@ -1,0 +1,283 @@
+/*
+ * LCKV decode-step attention: float64 CPU oracle.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, direct restatement of what
+ * the layer-condensed KV cache method computes at one decode step.  It exists
+ * to check the CUDA library and to be timed as a CPU baseline; the product
+ * path never calls it.  It shares no code, header, table or helper with the
+ * CUDA sources.
+ *
+ * Every function below states the passage of the paper (arXiv 2405.10637) it
+ * follows.  Arithmetic is float64 throughout; the bf16 inputs are widened
+ * exactly.  Softmax is the textbook two-pass form (max, then exponentials,
+ * then normalise): no chunking, no running rescale, no reordering.
+ *
+ * Pins (see tests/): brute-force n x n masked attention written independently
+ * in numpy, torch's scaled_dot_product_attention in float64 for w = L, closed
+ * forms (q = 0, one visible key, empty visible set, dominant key), permutation
+ * invariance, log-sum-exp merge of any partition, hand-enumerated warmup sets.
+ *
+ * Readings of the paper where it is silent (each one is a switch here):
+ *   top_variant 0  the shared cache is the cache of layer L-1 itself, even
+ *                  when that layer is a warmup layer (Section 2.1, literal);
+ *   top_variant 1  the shared cache is fed by the topmost non-warmup layer;
+ *   always_sink    0: the zero dummy key/value is used only when a query sees
+ *                  nothing (first token, Section 2.1); 1: it is a permanent
+ *                  extra column of every row (alternative reading, CPU only).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+#define LCKV_ORACLE_OK 0
+#define LCKV_ORACLE_EINVAL 1
+#define LCKV_ORACLE_ECAPACITY 2
+
+/* bf16 is the upper half of an IEEE binary32: widening is exact. */
+static double bf16_to_f64(uint16_t h)
+{
+    uint32_t u = ((uint32_t)h) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/*
+ * Layer plan.  Section 2.1: the top w/2 and the bottom w/2 layers are warmup
+ * layers with standard attention (sandwich); every other layer pairs its
+ * queries with the top layer's keys and values and drops the diagonal.
+ * "w = L" is the standard transformer (Section 4.2, the right-most point of
+ * the warmup-layer figure).
+ *
+ * Outputs, all of length L (layer 0 = bottom):
+ *   is_warmup[l]   1 if l is a warmup layer
+ *   read_slot[l]   which cache layer l attends to
+ *   mode[l]        0 = condensed (positions j <  t), 1 = standard (j <= t)
+ *   write_slot[l]  cache that receives layer l's new k,v (-1: layer has no K/V)
+ *   write_before[l] 1: the row is written before layer l attends (standard
+ *                  layers see their own token); 0: written at the end of the
+ *                  step (the shared cache under the diagonal mask)
+ * n_slots = number of distinct caches (the memory footprint in layers).
+ */
+int lckv_oracle_plan(int L, int w, int top_variant, int32_t* is_warmup, int32_t* read_slot,
+                     int32_t* mode, int32_t* write_slot, int32_t* write_before, int32_t* n_slots)
+{
+    if (L < 1 || w < 0 || w > L) return LCKV_ORACLE_EINVAL;
+    if (w != L && (w % 2) != 0) return LCKV_ORACLE_EINVAL;
+    if (top_variant != 0 && top_variant != 1) return LCKV_ORACLE_EINVAL;
+
+    for (int l = 0; l < L; ++l) {
+        if (w == L) is_warmup[l] = 1;
+        else is_warmup[l] = (l < w / 2) || (l >= L - w / 2);
+    }
+    /* which layer feeds the shared cache (slot 0) */
+    int feeder = L - 1;
+    if (top_variant == 1 && w > 0 && w < L) feeder = L - 1 - w / 2;
+
+    int next = 1;
+    for (int l = 0; l < L; ++l) {
+        if (is_warmup[l]) {
+            mode[l] = 1;
+            write_before[l] = 1;
+            if (l == feeder) {
+                read_slot[l] = write_slot[l] = 0;
+            } else {
+                read_slot[l] = write_slot[l] = next++;
+            }
+        } else {
+            mode[l] = 0;
+            read_slot[l] = 0;
+            write_before[l] = 0;
+            write_slot[l] = (l == feeder) ? 0 : -1;
+        }
+    }
+    *n_slots = next;
+    return LCKV_ORACLE_OK;
+}
+
+/*
+ * One query row against n_vis visible cache rows (Section 2.1):
+ *   s_j = scale * <q, K_j>,  p = softmax_j(s),  o = sum_j p_j V_j.
+ * An empty visible set is the first token of a sequence under the diagonal
+ * mask: it attends to one zero dummy key/value, which takes weight 1, so
+ * o = 0 (Section 2.1).  lse = log sum_j exp(s_j); for the empty set the dummy
+ * column has score 0, so lse = 0.
+ * probs (optional, n_vis + 1 entries) receives p_0..p_{n_vis-1} and, last, the
+ * weight of the dummy column (0 unless the set is empty or always_sink).
+ */
+static void attend_row(const uint16_t* q, const uint16_t* K, const uint16_t* V, int64_t n_vis,
+                       int d, double scale, int always_sink, double* o, double* lse,
+                       double* probs, double* scratch)
+{
+    int use_dummy = always_sink || n_vis == 0;
+    double M = use_dummy ? 0.0 : -INFINITY;
+    for (int64_t j = 0; j < n_vis; ++j) {
+        double s = 0.0;
+        for (int c = 0; c < d; ++c) s += bf16_to_f64(q[c]) * bf16_to_f64(K[j * d + c]);
+        s *= scale;
+        scratch[j] = s;
+        if (s > M) M = s;
+    }
+    double Z = use_dummy ? exp(0.0 - M) : 0.0;
+    for (int64_t j = 0; j < n_vis; ++j) {
+        scratch[j] = exp(scratch[j] - M);
+        Z += scratch[j];
+    }
+    for (int c = 0; c < d; ++c) o[c] = 0.0;
+    for (int64_t j = 0; j < n_vis; ++j) {
+        double p = scratch[j] / Z;
+        if (probs) probs[j] = p;
+        for (int c = 0; c < d; ++c) o[c] += p * bf16_to_f64(V[j * d + c]);
+    }
+    /* the dummy value is the zero vector: it adds nothing to o */
+    if (probs) probs[n_vis] = use_dummy ? exp(0.0 - M) / Z : 0.0;
+    if (lse) *lse = M + log(Z);
+}
+
+/* Single-row entry for tests: q[d], K,V [n_vis, d]. */
+int lckv_oracle_attend_row(const uint16_t* q, const uint16_t* K, const uint16_t* V,
+                           int64_t n_vis, int d, double scale, int always_sink, double* o,
+                           double* lse, double* probs)
+{
+    if (n_vis < 0 || d < 1) return LCKV_ORACLE_EINVAL;
+    double* scratch = (double*)malloc(sizeof(double) * (size_t)(n_vis > 0 ? n_vis : 1));
+    if (!scratch) return LCKV_ORACLE_EINVAL;
+    attend_row(q, K, V, n_vis, d, scale, always_sink, o, lse, probs, scratch);
+    free(scratch);
+    return LCKV_ORACLE_OK;
+}
+
+/*
+ * Batched decode attention of one layer against one cache.
+ *   q    [B, H_q, d]           bf16 bits
+ *   K, V [B, H_kv, T_cap, d]   bf16 bits, rows [0, n_vis) of each (b, kv head) valid
+ *   lens [B]                   tokens already cached; the new token is position lens[b]
+ *   mode 0: visible j < lens[b] (diagonal masked, Section 2.1)
+ *   mode 1: visible j <= lens[b] (standard attention of a warmup layer; row
+ *           lens[b] must already hold this step's k, v)
+ *   q head h reads kv head h / (H_q / H_kv)  (contiguous groups, Llama's GQA)
+ *   out [B, H_q, d] float64, lse [B, H_q] float64 (may be NULL)
+ * Rows are independent; they are spread over the host cores with OpenMP.
+ */
+int lckv_oracle_decode_attention(const uint16_t* q, const uint16_t* K, const uint16_t* V,
+                                 const int32_t* lens, int B, int H_q, int H_kv, int64_t T_cap,
+                                 int d, int mode, double scale, int always_sink, double* out,
+                                 double* lse)
+{
+    if (B < 0 || H_q < 1 || H_kv < 1 || H_q % H_kv != 0 || d < 1) return LCKV_ORACLE_EINVAL;
+    if (mode != 0 && mode != 1) return LCKV_ORACLE_EINVAL;
+    int g = H_q / H_kv;
+    for (int b = 0; b < B; ++b) {
+        if (lens[b] < 0 || (int64_t)lens[b] + mode > T_cap) return LCKV_ORACLE_ECAPACITY;
+    }
+    int64_t rows = (int64_t)B * H_q;
+#pragma omp parallel
+    {
+        double* scratch = (double*)malloc(sizeof(double) * (size_t)(T_cap > 0 ? T_cap : 1));
+#pragma omp for schedule(dynamic, 1)
+        for (int64_t r = 0; r < rows; ++r) {
+            int b = (int)(r / H_q), h = (int)(r % H_q);
+            int kvh = h / g;
+            int64_t n_vis = (int64_t)lens[b] + mode;
+            const uint16_t* Kp = K + (((int64_t)b * H_kv + kvh) * T_cap) * d;
+            const uint16_t* Vp = V + (((int64_t)b * H_kv + kvh) * T_cap) * d;
+            attend_row(q + r * d, Kp, Vp, n_vis, d, scale, always_sink, out + r * d,
+                       lse ? lse + r : NULL, NULL, scratch);
+        }
+        free(scratch);
+    }
+    return LCKV_ORACLE_OK;
+}
+
+/*
+ * Append: the new token's k, v (each [B, H_kv, d]) become row lens[b] of the
+ * cache (Section 1: the cache stores the keys and values of every generated
+ * token so they are not recomputed).  Lengths are not changed here.
+ */
+int lckv_oracle_append(uint16_t* K, uint16_t* V, const uint16_t* k_new, const uint16_t* v_new,
+                       const int32_t* lens, int B, int H_kv, int64_t T_cap, int d)
+{
+    for (int b = 0; b < B; ++b)
+        if (lens[b] < 0 || (int64_t)lens[b] >= T_cap) return LCKV_ORACLE_ECAPACITY;
+    for (int b = 0; b < B; ++b)
+        for (int h = 0; h < H_kv; ++h) {
+            int64_t dst = ((((int64_t)b * H_kv + h) * T_cap) + lens[b]) * d;
+            int64_t src = ((int64_t)b * H_kv + h) * d;
+            memcpy(K + dst, k_new + src, sizeof(uint16_t) * (size_t)d);
+            memcpy(V + dst, v_new + src, sizeof(uint16_t) * (size_t)d);
+        }
+    return LCKV_ORACLE_OK;
+}
+
+/*
+ * One decode step of the whole layer stack (Sections 2.1 and 2.2: decoding is
+ * one token at a time, bottom layer to top layer).  For l = 0 .. L-1 in order:
+ *   warmup layer:   write its k,v at row lens[b] of its own cache, then attend
+ *                   j <= lens[b]  (standard attention);
+ *   other layers:   attend j < lens[b] of the shared cache (the top layer's
+ *                   k,v of this token do not exist yet: diagonal masked).
+ * Then the feeder layer's k,v of this token are written at row lens[b] of the
+ * shared cache (unless it was a warmup layer that wrote them already) and
+ * every length grows by one.
+ *
+ *   q_layers[l]      [B, H_q, d]   one pointer per layer
+ *   k_new_layers[l], v_new_layers[l]   [B, H_kv, d] or NULL where write_slot[l] < 0
+ *   K_slots[s], V_slots[s]            [B_max, H_kv, T_cap, d] caches, modified
+ *   lens [B]                          modified (+1)
+ *   out_layers[l]    [B, H_q, d] float64; lse_layers[l] [B, H_q] or NULL array
+ */
+int lckv_oracle_stack_step(int L, int w, int top_variant, const uint16_t* const* q_layers,
+                           const uint16_t* const* k_new_layers,
+                           const uint16_t* const* v_new_layers, uint16_t* const* K_slots,
+                           uint16_t* const* V_slots, int32_t* lens, int B, int H_q, int H_kv,
+                           int64_t T_cap, int d, double scale, int always_sink,
+                           double* const* out_layers, double* const* lse_layers)
+{
+    int32_t* plan = (int32_t*)malloc(sizeof(int32_t) * 5 * (size_t)L);
+    if (!plan) return LCKV_ORACLE_EINVAL;
+    int32_t *is_w = plan, *rs = plan + L, *md = plan + 2 * L, *ws = plan + 3 * L,
+            *wb = plan + 4 * L;
+    int32_t n_slots = 0;
+    int rc = lckv_oracle_plan(L, w, top_variant, is_w, rs, md, ws, wb, &n_slots);
+    if (rc) { free(plan); return rc; }
+    for (int b = 0; b < B; ++b)
+        if (lens[b] < 0 || (int64_t)lens[b] + 1 > T_cap) { free(plan); return LCKV_ORACLE_ECAPACITY; }
+    for (int l = 0; l < L; ++l)
+        if (ws[l] >= 0 && (!k_new_layers[l] || !v_new_layers[l])) { free(plan); return LCKV_ORACLE_EINVAL; }
+
+    for (int l = 0; l < L && rc == 0; ++l) {
+        if (ws[l] >= 0 && wb[l])
+            rc = lckv_oracle_append(K_slots[ws[l]], V_slots[ws[l]], k_new_layers[l],
+                                    v_new_layers[l], lens, B, H_kv, T_cap, d);
+        if (rc) break;
+        rc = lckv_oracle_decode_attention(q_layers[l], K_slots[rs[l]], V_slots[rs[l]], lens, B,
+                                          H_q, H_kv, T_cap, d, md[l], scale, always_sink,
+                                          out_layers[l], lse_layers ? lse_layers[l] : NULL);
+    }
+    for (int l = 0; l < L && rc == 0; ++l)
+        if (ws[l] >= 0 && !wb[l])
+            rc = lckv_oracle_append(K_slots[ws[l]], V_slots[ws[l]], k_new_layers[l],
+                                    v_new_layers[l], lens, B, H_kv, T_cap, d);
+    if (rc == 0)
+        for (int b = 0; b < B; ++b) lens[b] += 1;
+    free(plan);
+    return rc;
+}
+
+/* Threads the parallel loops use (reported beside the CPU baseline). */
+int lckv_oracle_num_threads(void)
+{
+    int n = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+    {
+#pragma omp single
+        n = omp_get_num_threads();
+    }
+#endif
+    return n;
+}

@@ -1,0 +1,158 @@
+"""ctypes/numpy front end of the float64 CPU oracle (oracle/lckv_oracle.c).
+
+TEST INFRASTRUCTURE ONLY: imported by tests/, by the smoke check and by the
+CPU-baseline leg of the benchmark.  Nothing here touches CUDA, and the CUDA
+package never imports this module.
+
+bf16 tensors travel as numpy uint16 arrays holding the raw bits.
+"""
+import ctypes as C
+import os
+
+import numpy as np
+
+from . import build as _build
+
+_LIB = None
+
+
+def lib():
+    global _LIB
+    if _LIB is None:
+        path = _build.build()
+        L = C.CDLL(path)
+        u16p, i32p, f64p = C.POINTER(C.c_uint16), C.POINTER(C.c_int32), C.POINTER(C.c_double)
+        L.lckv_oracle_plan.argtypes = [C.c_int, C.c_int, C.c_int] + [i32p] * 6
+        L.lckv_oracle_plan.restype = C.c_int
+        L.lckv_oracle_attend_row.argtypes = [u16p, u16p, u16p, C.c_int64, C.c_int, C.c_double,
+                                             C.c_int, f64p, f64p, f64p]
+        L.lckv_oracle_attend_row.restype = C.c_int
+        L.lckv_oracle_decode_attention.argtypes = [u16p, u16p, u16p, i32p, C.c_int, C.c_int,
+                                                   C.c_int, C.c_int64, C.c_int, C.c_int,
+                                                   C.c_double, C.c_int, f64p, f64p]
+        L.lckv_oracle_decode_attention.restype = C.c_int
+        L.lckv_oracle_append.argtypes = [u16p, u16p, u16p, u16p, i32p, C.c_int, C.c_int,
+                                         C.c_int64, C.c_int]
+        L.lckv_oracle_append.restype = C.c_int
+        pp = C.POINTER(C.c_void_p)
+        L.lckv_oracle_stack_step.argtypes = [C.c_int, C.c_int, C.c_int, pp, pp, pp, pp, pp, i32p,
+                                             C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int,
+                                             C.c_double, C.c_int, pp, pp]
+        L.lckv_oracle_stack_step.restype = C.c_int
+        L.lckv_oracle_num_threads.restype = C.c_int
+        _LIB = L
+    return _LIB
+
+
+class OracleError(RuntimeError):
+    pass
+
+
+def _chk(rc, what):
+    if rc != 0:
+        raise OracleError(f"{what}: oracle status {rc} ({ {1: 'EINVAL', 2: 'ECAPACITY'}.get(rc, '?') })")
+
+
+def _u16(a):
+    a = np.ascontiguousarray(a)
+    assert a.dtype == np.uint16, a.dtype
+    return a
+
+
+def _p(a, ct):
+    return a.ctypes.data_as(C.POINTER(ct))
+
+
+def num_threads():
+    return int(lib().lckv_oracle_num_threads())
+
+
+def plan(L, w, top_variant=0):
+    """Layer plan (Section 2.1 sandwich rule).  Returns a dict of int32 arrays + n_slots."""
+    arrs = [np.zeros(L, np.int32) for _ in range(5)]
+    n = np.zeros(1, np.int32)
+    rc = lib().lckv_oracle_plan(L, w, top_variant, *[_p(a, C.c_int32) for a in arrs],
+                                _p(n, C.c_int32))
+    _chk(rc, "plan")
+    keys = ["is_warmup", "read_slot", "mode", "write_slot", "write_before"]
+    out = dict(zip(keys, arrs))
+    out["n_slots"] = int(n[0])
+    return out
+
+
+def attend_row(q, K, V, scale, always_sink=False, want_probs=False):
+    """One query q[d] against K,V [n, d] (uint16 bf16 bits).  Returns (o, lse[, probs])."""
+    q, K, V = _u16(q), _u16(K), _u16(V)
+    d = q.shape[-1]
+    n = K.shape[0] if K.size else 0
+    o = np.zeros(d, np.float64)
+    lse = np.zeros(1, np.float64)
+    probs = np.zeros(n + 1, np.float64)
+    rc = lib().lckv_oracle_attend_row(_p(q, C.c_uint16), _p(K, C.c_uint16), _p(V, C.c_uint16),
+                                      n, d, float(scale), int(always_sink), _p(o, C.c_double),
+                                      _p(lse, C.c_double), _p(probs, C.c_double))
+    _chk(rc, "attend_row")
+    return (o, float(lse[0]), probs) if want_probs else (o, float(lse[0]))
+
+
+def decode_attention(q, K, V, lens, mode, scale, always_sink=False):
+    """q [B,Hq,d], K,V [B,Hkv,Tcap,d] uint16, lens [B] int32 -> (out [B,Hq,d], lse [B,Hq]) float64."""
+    q, K, V = _u16(q), _u16(K), _u16(V)
+    lens = np.ascontiguousarray(lens, np.int32)
+    B, Hq, d = q.shape
+    _, Hkv, Tcap, _ = K.shape
+    assert K.shape[0] >= B and V.shape == K.shape
+    out = np.zeros((B, Hq, d), np.float64)
+    lse = np.zeros((B, Hq), np.float64)
+    rc = lib().lckv_oracle_decode_attention(_p(q, C.c_uint16), _p(K, C.c_uint16),
+                                            _p(V, C.c_uint16), _p(lens, C.c_int32), B, Hq, Hkv,
+                                            Tcap, d, int(mode), float(scale), int(always_sink),
+                                            _p(out, C.c_double), _p(lse, C.c_double))
+    _chk(rc, "decode_attention")
+    return out, lse
+
+
+def append(K, V, k_new, v_new, lens):
+    """In place: row lens[b] of K,V [B,Hkv,Tcap,d] <- k_new, v_new [B,Hkv,d]."""
+    assert K.flags.c_contiguous and V.flags.c_contiguous and K.dtype == np.uint16
+    k_new, v_new = _u16(k_new), _u16(v_new)
+    lens = np.ascontiguousarray(lens, np.int32)
+    B, Hkv, d = k_new.shape
+    rc = lib().lckv_oracle_append(_p(K, C.c_uint16), _p(V, C.c_uint16), _p(k_new, C.c_uint16),
+                                  _p(v_new, C.c_uint16), _p(lens, C.c_int32), B, Hkv,
+                                  K.shape[2], d)
+    _chk(rc, "append")
+
+
+def _ptr_array(arrs):
+    t = (C.c_void_p * len(arrs))()
+    for i, a in enumerate(arrs):
+        t[i] = None if a is None else a.ctypes.data
+    return C.cast(t, C.POINTER(C.c_void_p))
+
+
+def stack_step(L, w, q_layers, k_new_layers, v_new_layers, K_slots, V_slots, lens, scale,
+               top_variant=0, always_sink=False):
+    """One decode step of the whole stack; caches and lens are updated in place.
+
+    q_layers: list of L arrays [B,Hq,d]; k_new_layers/v_new_layers: list of L arrays
+    [B,Hkv,d] or None; K_slots/V_slots: list of caches [Bmax,Hkv,Tcap,d]; lens int32 [B].
+    Returns (outs, lses): lists of L float64 arrays.
+    """
+    q_layers = [_u16(q) for q in q_layers]
+    k_new_layers = [None if k is None else _u16(k) for k in k_new_layers]
+    v_new_layers = [None if v is None else _u16(v) for v in v_new_layers]
+    for a in list(K_slots) + list(V_slots):
+        assert a.flags.c_contiguous and a.dtype == np.uint16
+    assert lens.dtype == np.int32 and lens.flags.c_contiguous
+    B, Hq, d = q_layers[0].shape
+    _, Hkv, Tcap, _ = K_slots[0].shape
+    outs = [np.zeros((B, Hq, d), np.float64) for _ in range(L)]
+    lses = [np.zeros((B, Hq), np.float64) for _ in range(L)]
+    rc = lib().lckv_oracle_stack_step(L, w, int(top_variant), _ptr_array(q_layers),
+                                      _ptr_array(k_new_layers), _ptr_array(v_new_layers),
+                                      _ptr_array(K_slots), _ptr_array(V_slots),
+                                      _p(lens, C.c_int32), B, Hq, Hkv, Tcap, d, float(scale),
+                                      int(always_sink), _ptr_array(outs), _ptr_array(lses))
+    _chk(rc, "stack_step")
+    return outs, lses
