@@ -1,0 +1,236 @@
+/*
+ * lckv.h - C ABI of the B200 (sm_100a) decode-step attention library for the
+ * Layer-Condensed KV Cache (LCKV, arXiv 2405.10637).
+ *
+ * What the library computes (paper, Section 2.1).  In an LCKV decoder the
+ * queries of every non-warmup layer are paired with the keys and values of
+ * the TOP layer only, so one cache is shared by all those layers; a token does
+ * not attend to itself there (the diagonal of the attention matrix is masked,
+ * because the top layer's k,v of the current token do not exist yet while the
+ * lower layers run), and a token that sees nothing attends to a zero dummy
+ * key/value, i.e. its output is the zero vector.  The top w/2 and bottom w/2
+ * layers ("warmup layers", sandwich placement) keep standard attention over
+ * their own per-layer caches, including the current token.  Decoding proceeds
+ * one token at a time, bottom layer to top layer (Section 2.2).
+ *
+ * Conventions common to every call
+ *   - All tensor arguments are DEVICE pointers unless a name says "host".
+ *   - bf16 tensors are raw 16-bit patterns (upper half of IEEE binary32),
+ *     contiguous, 16-byte aligned.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default
+ *     stream).  Calls only enqueue work; none synchronises unless it says so.
+ *   - The library allocates no device memory: the caller hands one device
+ *     buffer to lckv_cache_alloc and keeps it alive until lckv_cache_free.
+ *   - Every call returns an int status (LCKV_OK = 0).  Nothing aborts, throws
+ *     or traps.  On any non-zero status nothing was enqueued and no length
+ *     changed, unless stated otherwise.
+ *   - A cache object is not thread-safe; use it from one host thread and one
+ *     stream at a time (kernels of one cache share its workspace).
+ */
+#ifndef LCKV_H
+#define LCKV_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+enum {
+    LCKV_OK = 0,
+    LCKV_EINVAL = 1,    /* null pointer, bad shape, odd w, batch > max_batch, bad slot or mode  */
+    LCKV_ECAPACITY = 2, /* a sequence would exceed max_seq rows                                */
+    LCKV_ENOMEM = 3,    /* caller's buffer too small or not 256-byte aligned                   */
+    LCKV_ECUDA = 4,     /* a CUDA runtime/driver call failed; see lckv_last_cuda_error         */
+    LCKV_ETIMEOUT = 5   /* a bounded device-side wait gave up (reported by lckv_cache_status)  */
+};
+
+enum {
+    LCKV_MODE_CONDENSED = 0, /* visible positions j <  len[b]: diagonal masked (Section 2.1) */
+    LCKV_MODE_STANDARD = 1   /* visible positions j <= len[b]: warmup layers  (Section 2.1)  */
+};
+
+typedef struct lckv_cache lckv_cache_t; /* opaque host object */
+
+/* Plain-old-data description of a layer stack and its caches. */
+typedef struct {
+    uint32_t struct_size;  /* sizeof(lckv_config_t), for versioning                          */
+    int32_t n_layers;      /* L >= 1, layer 0 = bottom                                       */
+    int32_t n_warmup;      /* w: even with 0 <= w < L, or w == L (standard transformer)      */
+    int32_t n_q_heads;     /* H_q                                                            */
+    int32_t n_kv_heads;    /* H_kv, H_q % H_kv == 0; q head h reads kv head h / (H_q/H_kv)   */
+    int32_t head_dim;      /* d_h: 64 or 128                                                 */
+    int32_t max_batch;     /* B_max >= 1                                                     */
+    int32_t max_seq;       /* T_cap >= 1 rows per sequence per cache                         */
+    float softmax_scale;   /* 0 => 1/sqrt(d_h)                                               */
+    int32_t top_variant;   /* which layer feeds the shared cache, see lckv_plan              */
+    int32_t out_dtype;     /* 0 = bf16 outputs, 1 = fp32 outputs                             */
+    int32_t host_staging;  /* 1: reserve device staging for lckv_layer_stack_step_host       */
+    int32_t use_graph;     /* 1: lckv_layer_stack_step replays a CUDA graph when the argument
+                              pointers repeat from the previous call                         */
+    int32_t kernel_kind;   /* 0 = choose (tensor-core kernel when the query group is a dense
+                              MMA tile, else the FP32-ALU kernel); 1 = force FP32-ALU        */
+} lckv_config_t;
+
+/* Facts about a built cache that a caller or a benchmark may want. */
+typedef struct {
+    int32_t n_slots;          /* distinct caches held (footprint in layers)                  */
+    int32_t n_workers;        /* independent workers (warps) per attention launch            */
+    int32_t rows_per_tile;    /* cache rows moved by one bulk copy                           */
+    int32_t kernel_kind;      /* 1 = FP32-ALU kernel (one q head per pair),
+                                 2 = tensor-core kernel (one kv head's query group per pair) */
+    int32_t launches_per_step;/* kernels lckv_layer_stack_step enqueues                      */
+    int32_t sm_count;
+    uint64_t slot_bytes;      /* bytes of one K (or V) tensor of one slot                    */
+    uint64_t workspace_bytes; /* lengths + plan tables + split-K partials + counters         */
+} lckv_info_t;
+
+/*
+ * Layer plan (Section 2.1: the top w/2 layers and the bottom w/2 layers are
+ * warmup layers; Section 4.2: w = L is the standard transformer).  Host only,
+ * no GPU needed.  All output arrays have n_layers entries.
+ *   is_warmup[l]     1 for warmup layers
+ *   read_slot[l]     cache slot layer l attends to (slot 0 = the shared top-layer cache)
+ *   mode[l]          LCKV_MODE_CONDENSED or LCKV_MODE_STANDARD
+ *   write_slot[l]    slot that receives layer l's new k,v, or -1 (layer computes no K/V)
+ *   write_before[l]  1: appended before layer l attends (standard layers see
+ *                    their own token); 0: appended at the end of the step
+ * top_variant 0 (paper-literal): slot 0 is the cache of layer L-1 itself; if
+ *   that layer is a warmup layer it uses slot 0 with standard attention while
+ *   the condensed layers below it see slot 0 without the current token.
+ *   Footprint max(w,1) caches.
+ * top_variant 1: slot 0 is fed by the topmost non-warmup layer L-1-w/2 and the
+ *   w warmup layers own slots 1..w.  Footprint min(w+1, L) caches.
+ * Errors: LCKV_EINVAL for null pointers, L < 1, odd w, w > L, bad variant.
+ */
+int lckv_plan(int32_t n_layers, int32_t n_warmup, int32_t top_variant, int32_t* is_warmup,
+              int32_t* read_slot, int32_t* mode, int32_t* write_slot, int32_t* write_before,
+              int32_t* n_slots);
+
+/*
+ * Device bytes lckv_cache_alloc needs for this configuration (caches for every
+ * slot of the plan + lengths + workspace + optional staging), or 0 if the
+ * configuration is invalid.  Needs a CUDA device (the workspace is sized from
+ * the SM count of the current device).
+ */
+size_t lckv_cache_bytes(const lckv_config_t* cfg);
+
+/*
+ * Build a cache object over caller-owned device memory (Section 1: the KV
+ * cache stores each layer's keys and values of past tokens; here only
+ * max(w,1) or w+1 layers have one).
+ *   dev_buf/dev_bytes  device buffer, 256-byte aligned, >= lckv_cache_bytes(cfg).
+ *                      The caller owns it; the library never frees it.
+ * Layout inside: per slot one K and one V tensor [B_max, H_kv, T_cap, d_h]
+ * bf16, contiguous; one int32 length per sequence shared by all slots (all
+ * caches advance together).  Lengths start at 0 and the workspace is cleared
+ * (this call synchronises the device once).  Cache contents are NOT cleared.
+ * Errors: EINVAL (bad config / null), ENOMEM (buffer small or misaligned),
+ * ECUDA.
+ */
+int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf,
+                     size_t dev_bytes);
+
+/* Destroys the host object (and any CUDA graph it holds).  The device buffer stays the caller's. */
+int lckv_cache_free(lckv_cache_t* cache);
+
+/* Fills *info.  EINVAL on null. */
+int lckv_cache_info(const lckv_cache_t* cache, lckv_info_t* info);
+
+/*
+ * Set per-sequence lengths (tokens already cached) from a HOST array, or all to
+ * zero if host_lens is NULL; clears the split-K workspace and the device
+ * status word.  Enqueued on `stream`; host_lens may be reused on return.
+ * Errors: EINVAL (batch out of range, negative length), ECAPACITY (a length
+ * > T_cap), ECUDA.
+ */
+int lckv_cache_reset(lckv_cache_t* cache, const int32_t* host_lens, int32_t batch, void* stream);
+
+/* Copies the device lengths of the first `batch` sequences to host_out; SYNCHRONISES `stream`. */
+int lckv_cache_lengths(const lckv_cache_t* cache, int32_t* host_out, int32_t batch, void* stream);
+
+/*
+ * Reads the device status word (0, or LCKV_ETIMEOUT if some kernel's bounded
+ * wait on a copy gave up; the outputs of that launch are then undefined);
+ * SYNCHRONISES `stream`.  lckv_cache_reset clears it.
+ */
+int lckv_cache_status(const lckv_cache_t* cache, int32_t* host_status, void* stream);
+
+/* Device pointers of slot `slot`'s K and V tensors [B_max, H_kv, T_cap, d_h] bf16 (for filling
+ * a cache with a prompt's keys and values, or inspecting it).  EINVAL on bad slot / null. */
+int lckv_cache_slot_ptrs(const lckv_cache_t* cache, int32_t slot, void** k, void** v);
+
+/*
+ * Append (Section 2.1: only the top layer and the warmup layers compute K/V):
+ * writes k_new, v_new [batch, H_kv, d_h] bf16 as row len[b] of slot `slot` for
+ * every b < batch; bit-exact copy.  If advance_len != 0 every len[b], b < batch,
+ * grows by one afterwards (this advances ALL slots: they share the lengths).
+ * Errors: EINVAL, ECAPACITY (some len[b] + 1 > T_cap, judged from the host
+ * mirror of the lengths; nothing written), ECUDA.
+ */
+int lckv_append_kv(lckv_cache_t* cache, int32_t slot, const void* k_new, const void* v_new,
+                   int32_t batch, int32_t advance_len, void* stream);
+
+/*
+ * Decode attention of one layer for one new token per sequence (Section 2.1):
+ *   out[b,h] = sum_j softmax_j( scale * <q[b,h], K[b,kv(h),j]> ) * V[b,kv(h),j]
+ * over the visible rows j of slot `slot`: j < len[b] (LCKV_MODE_CONDENSED,
+ * diagonal masked) or j <= len[b] (LCKV_MODE_STANDARD; row len[b] must have
+ * been appended without advancing).  A row that sees nothing (condensed mode,
+ * len[b] == 0) gets the zero vector (zero dummy key/value) and lse 0.
+ *   q    [batch, H_q, d_h] bf16
+ *   out  [batch, H_q, d_h] bf16 (or fp32 if out_dtype == 1)
+ *   lse  [batch, H_q] fp32 natural-log sum of exponentials of the scaled
+ *        scores, or NULL
+ * Arithmetic: fp32 scores, fp32 running max / sum / accumulators, split over
+ * the sequence with a log-sum-exp merge of fp32 partials, one rounding to the
+ * output type.  Rows >= the visible count are never read.
+ * Errors: EINVAL, ECAPACITY (mode STANDARD with a full sequence), ECUDA.
+ */
+int lckv_decode_attention(lckv_cache_t* cache, int32_t slot, int32_t mode, const void* q,
+                          void* out, float* lse, int32_t batch, void* stream);
+
+/*
+ * One decode step of the whole layer stack (Sections 2.1, 2.2), layers in
+ * order as DEPENDENT launches on `stream` - layer l+1's query is a function of
+ * layer l's output in a real model, so queries of different layers are never
+ * batched into one pass.  For l = 0..L-1, following lckv_plan:
+ *   write_before[l]: append k_new_layers[l], v_new_layers[l] to write_slot[l];
+ *   attend q_layers[l] over read_slot[l] in mode[l] into out_layers[l];
+ * then append the feeder layer's k,v to slot 0 if not done yet, then
+ * len[b] += 1 for b < batch.
+ *   q_layers, out_layers            HOST arrays of L device pointers
+ *   k_new_layers, v_new_layers      HOST arrays of L device pointers; entries of
+ *                                   layers with write_slot[l] < 0 are ignored
+ * Errors: EINVAL (null array, null required entry, batch), ECAPACITY (some
+ * sequence is full; nothing enqueued), ECUDA.
+ */
+int lckv_layer_stack_step(lckv_cache_t* cache, const void* const* q_layers,
+                          void* const* out_layers, const void* const* k_new_layers,
+                          const void* const* v_new_layers, int32_t batch, void* stream);
+
+/*
+ * The same step for callers whose activations live in HOST memory (pinned for
+ * real overlap): copies every layer's q (and the k,v of layers that have them)
+ * host->device into the cache's staging area, runs the step, copies every
+ * layer's output device->host.  All on `stream`, asynchronous; synchronise the
+ * stream before reading the outputs.  Needs host_staging = 1 at alloc.
+ * Array arguments are HOST arrays of L HOST pointers with the shapes above.
+ */
+int lckv_layer_stack_step_host(lckv_cache_t* cache, const void* const* q_layers_host,
+                               void* const* out_layers_host,
+                               const void* const* k_new_layers_host,
+                               const void* const* v_new_layers_host, int32_t batch,
+                               void* stream);
+
+/* Short English name of a status code. */
+const char* lckv_status_string(int status);
+
+/* cudaError_t (as int) of the last failed CUDA call made by this library on this thread. */
+int lckv_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* LCKV_H */

@@ -1,0 +1,497 @@
+// Host runtime and C ABI of the LCKV decode-attention library (see include/lckv.h).
+#include <cuda_runtime.h>
+
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <vector>
+
+#include "../../include/lckv.h"
+#include "lckv_attn_alu.cuh"
+#include "lckv_small_kernels.cuh"
+
+namespace {
+
+thread_local int g_last_cuda_error = 0;
+
+inline bool cuda_ok(cudaError_t e)
+{
+    if (e != cudaSuccess) {
+        g_last_cuda_error = (int)e;
+        return false;
+    }
+    return true;
+}
+
+inline size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+// Host-side layer plan; the rule is stated in the header (Section 2.1 of the paper).
+struct Plan {
+    std::vector<int32_t> is_warmup, read_slot, mode, write_slot, write_before;
+    int32_t n_slots = 0;
+};
+
+int make_plan(int L, int w, int variant, Plan& pl)
+{
+    if (L < 1 || w < 0 || w > L) return LCKV_EINVAL;
+    if (w != L && (w & 1)) return LCKV_EINVAL;
+    if (variant != 0 && variant != 1) return LCKV_EINVAL;
+    pl.is_warmup.assign(L, 0);
+    pl.read_slot.assign(L, 0);
+    pl.mode.assign(L, LCKV_MODE_CONDENSED);
+    pl.write_slot.assign(L, -1);
+    pl.write_before.assign(L, 0);
+    const int half = w / 2;
+    for (int l = 0; l < L; ++l) pl.is_warmup[l] = (w == L) || l < half || l >= L - half;
+    // The layer whose k,v fill slot 0.
+    const int feeder = (variant == 1 && w > 0 && w < L) ? L - 1 - half : L - 1;
+    int next_slot = 1;
+    for (int l = 0; l < L; ++l) {
+        if (pl.is_warmup[l]) {
+            const int s = (l == feeder) ? 0 : next_slot++;
+            pl.read_slot[l] = pl.write_slot[l] = s;
+            pl.mode[l] = LCKV_MODE_STANDARD;
+            pl.write_before[l] = 1;
+        } else if (l == feeder) {
+            pl.write_slot[l] = 0;
+        }
+    }
+    pl.n_slots = next_slot;
+    return LCKV_OK;
+}
+
+struct Layout {
+    size_t off_lens, off_pre, off_start, off_counters, off_status, off_partials, off_slots;
+    size_t off_stage_q, off_stage_out, off_stage_kv;
+    size_t slot_bytes, workspace_bytes, total_bytes;
+    size_t stage_q_bytes, stage_out_bytes, stage_kv_bytes;  // per layer
+    int pre_stride;
+};
+
+}  // namespace
+
+struct lckv_cache {
+    lckv_config_t cfg;
+    Plan plan;
+    Layout lay;
+    float scale_log2;
+    int sm_count, n_workers, grid, rows_per_tile, h_pairs, kernel_kind;
+    uint8_t* base;
+    int32_t* d_lens;
+    uint32_t* d_pre;
+    int32_t* d_start;
+    int32_t* d_counters;
+    int32_t* d_status;
+    float* d_partials;
+    std::vector<int32_t> h_lens;  // host mirror of the device lengths
+    int n_kv_layers;
+};
+
+namespace {
+
+int validate_config(const lckv_config_t* c)
+{
+    if (!c || c->struct_size != sizeof(lckv_config_t)) return LCKV_EINVAL;
+    if (c->n_layers < 1 || c->n_q_heads < 1 || c->n_kv_heads < 1) return LCKV_EINVAL;
+    if (c->n_q_heads % c->n_kv_heads) return LCKV_EINVAL;
+    if (c->head_dim != 64 && c->head_dim != 128) return LCKV_EINVAL;
+    if (c->max_batch < 1 || c->max_seq < 1) return LCKV_EINVAL;
+    if (!(c->softmax_scale >= 0.f) || !std::isfinite(c->softmax_scale)) return LCKV_EINVAL;
+    if (c->out_dtype != 0 && c->out_dtype != 1) return LCKV_EINVAL;
+    if (c->kernel_kind != 0 && c->kernel_kind != 1) return LCKV_EINVAL;
+    Plan pl;
+    if (int rc = make_plan(c->n_layers, c->n_warmup, c->top_variant, pl)) return rc;
+    // tile counts are kept in 32 bits
+    const uint64_t tiles = (uint64_t)c->max_batch * (((uint64_t)c->max_seq + 15) / 16);
+    if (tiles >= (1ull << 31)) return LCKV_EINVAL;
+    return LCKV_OK;
+}
+
+int resolve_kernel_kind(const lckv_config_t&) { return 1; }
+
+void make_layout(const lckv_config_t& c, int n_slots, int n_workers, int n_kv_layers, Layout& y)
+{
+    const size_t A = 256;
+    size_t off = 0;
+    y.off_lens = off;      off = align_up(off + (size_t)c.max_batch * 4, A);
+    y.pre_stride = (int)align_up((size_t)c.max_batch + 1, 64);
+    y.off_pre = off;       off = align_up(off + 2 * (size_t)y.pre_stride * 4, A);
+    y.off_start = off;     off = align_up(off + 2 * (size_t)n_workers * 4, A);
+    y.off_counters = off;  off = align_up(off + (size_t)n_workers * 4, A);
+    y.off_status = off;    off = align_up(off + 4, A);
+    y.off_partials = off;  off = align_up(off + 2 * (size_t)n_workers * (c.head_dim + 4) * 4, A);
+    y.workspace_bytes = off;
+    y.slot_bytes =
+        align_up((size_t)c.max_batch * c.n_kv_heads * (size_t)c.max_seq * c.head_dim * 2, A);
+    y.off_slots = off;     off += 2 * (size_t)n_slots * y.slot_bytes;
+    y.stage_q_bytes = align_up((size_t)c.max_batch * c.n_q_heads * c.head_dim * 2, A);
+    y.stage_out_bytes =
+        align_up((size_t)c.max_batch * c.n_q_heads * c.head_dim * (c.out_dtype ? 4 : 2), A);
+    y.stage_kv_bytes = align_up((size_t)c.max_batch * c.n_kv_heads * c.head_dim * 2, A);
+    y.off_stage_q = y.off_stage_out = y.off_stage_kv = 0;
+    if (c.host_staging) {
+        y.off_stage_q = off;    off += (size_t)c.n_layers * y.stage_q_bytes;
+        y.off_stage_out = off;  off += (size_t)c.n_layers * y.stage_out_bytes;
+        y.off_stage_kv = off;   off += 2 * (size_t)n_kv_layers * y.stage_kv_bytes;
+    }
+    y.total_bytes = off;
+}
+
+int device_sm_count(int* sm)
+{
+    int dev = 0;
+    if (!cuda_ok(cudaGetDevice(&dev))) return LCKV_ECUDA;
+    if (!cuda_ok(cudaDeviceGetAttribute(sm, cudaDevAttrMultiProcessorCount, dev))) return LCKV_ECUDA;
+    return LCKV_OK;
+}
+
+uint16_t* slot_k(const lckv_cache* c, int s)
+{
+    return reinterpret_cast<uint16_t*>(c->base + c->lay.off_slots + (size_t)(2 * s) * c->lay.slot_bytes);
+}
+uint16_t* slot_v(const lckv_cache* c, int s)
+{
+    return reinterpret_cast<uint16_t*>(c->base + c->lay.off_slots +
+                                       (size_t)(2 * s + 1) * c->lay.slot_bytes);
+}
+
+int max_len(const lckv_cache* c, int batch)
+{
+    int m = 0;
+    for (int b = 0; b < batch; ++b) m = c->h_lens[b] > m ? c->h_lens[b] : m;
+    return m;
+}
+
+int launch_plan(lckv_cache* c, int batch, cudaStream_t st)
+{
+    lckv::plan_kernel<<<1, 1024, 0, st>>>(c->d_lens, batch, c->rows_per_tile, c->h_pairs,
+                                          c->n_workers, c->d_pre, c->lay.pre_stride, c->d_start);
+    return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
+}
+
+int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out, float* lse,
+                     int batch, cudaStream_t st)
+{
+    lckv::AttnParams p;
+    p.K = slot_k(c, slot);
+    p.V = slot_v(c, slot);
+    p.q = static_cast<const uint16_t*>(q);
+    p.out = out;
+    p.lse = lse;
+    p.lens = c->d_lens;
+    p.pre = c->d_pre + (size_t)mode * c->lay.pre_stride;
+    p.start_b = c->d_start + (size_t)mode * c->n_workers;
+    p.partials = c->d_partials;
+    p.counters = c->d_counters;
+    p.status = c->d_status;
+    p.T_cap = c->cfg.max_seq;
+    p.B = batch;
+    p.H_q = c->cfg.n_q_heads;
+    p.H_kv = c->cfg.n_kv_heads;
+    p.mode = mode;
+    p.n_workers = c->n_workers;
+    p.out_f32 = c->cfg.out_dtype;
+    p.scale_log2 = c->scale_log2;
+    if (c->cfg.head_dim == 128)
+        lckv::attn_alu_kernel<128><<<c->grid, lckv::kAluWarps * 32, lckv::kAluSmemBytes, st>>>(p);
+    else
+        lckv::attn_alu_kernel<64><<<c->grid, lckv::kAluWarps * 32, lckv::kAluSmemBytes, st>>>(p);
+    return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
+}
+
+int launch_append(lckv_cache* c, int slot, const void* k_new, const void* v_new, int batch,
+                  cudaStream_t st)
+{
+    const int64_t n = (int64_t)batch * c->cfg.n_kv_heads * (c->cfg.head_dim / 8);
+    const int threads = 256;
+    const int blocks = (int)((n + threads - 1) / threads);
+    lckv::append_kernel<<<blocks, threads, 0, st>>>(
+        slot_k(c, slot), slot_v(c, slot), static_cast<const uint16_t*>(k_new),
+        static_cast<const uint16_t*>(v_new), c->d_lens, batch, c->cfg.n_kv_heads, c->cfg.max_seq,
+        c->cfg.head_dim);
+    return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
+}
+
+int launch_advance(lckv_cache* c, int batch, cudaStream_t st)
+{
+    lckv::advance_kernel<<<(batch + 255) / 256, 256, 0, st>>>(c->d_lens, batch);
+    if (!cuda_ok(cudaGetLastError())) return LCKV_ECUDA;
+    for (int b = 0; b < batch; ++b) c->h_lens[b] += 1;
+    return LCKV_OK;
+}
+
+// The launches of one step, in the order the header states.
+int enqueue_step(lckv_cache* c, const void* const* q, void* const* out, const void* const* kn,
+                 const void* const* vn, int batch, cudaStream_t st)
+{
+    const Plan& pl = c->plan;
+    const int L = c->cfg.n_layers;
+    if (int rc = launch_plan(c, batch, st)) return rc;
+    for (int l = 0; l < L; ++l) {
+        if (pl.write_slot[l] >= 0 && pl.write_before[l])
+            if (int rc = launch_append(c, pl.write_slot[l], kn[l], vn[l], batch, st)) return rc;
+        if (int rc = launch_attention(c, pl.read_slot[l], pl.mode[l], q[l], out[l], nullptr, batch, st))
+            return rc;
+    }
+    for (int l = 0; l < L; ++l)
+        if (pl.write_slot[l] >= 0 && !pl.write_before[l])
+            if (int rc = launch_append(c, pl.write_slot[l], kn[l], vn[l], batch, st)) return rc;
+    return launch_advance(c, batch, st);
+}
+
+}  // namespace
+
+extern "C" {
+
+int lckv_plan(int32_t n_layers, int32_t n_warmup, int32_t top_variant, int32_t* is_warmup,
+              int32_t* read_slot, int32_t* mode, int32_t* write_slot, int32_t* write_before,
+              int32_t* n_slots)
+{
+    if (!is_warmup || !read_slot || !mode || !write_slot || !write_before || !n_slots)
+        return LCKV_EINVAL;
+    Plan pl;
+    if (int rc = make_plan(n_layers, n_warmup, top_variant, pl)) return rc;
+    for (int l = 0; l < n_layers; ++l) {
+        is_warmup[l] = pl.is_warmup[l];
+        read_slot[l] = pl.read_slot[l];
+        mode[l] = pl.mode[l];
+        write_slot[l] = pl.write_slot[l];
+        write_before[l] = pl.write_before[l];
+    }
+    *n_slots = pl.n_slots;
+    return LCKV_OK;
+}
+
+size_t lckv_cache_bytes(const lckv_config_t* cfg)
+{
+    if (validate_config(cfg)) return 0;
+    int sm = 0;
+    if (device_sm_count(&sm)) return 0;
+    Plan pl;
+    make_plan(cfg->n_layers, cfg->n_warmup, cfg->top_variant, pl);
+    int n_kv = 0;
+    for (int l = 0; l < cfg->n_layers; ++l) n_kv += pl.write_slot[l] >= 0;
+    Layout y;
+    make_layout(*cfg, pl.n_slots, sm * lckv::kAluWarps, n_kv, y);
+    return y.total_bytes;
+}
+
+int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf, size_t dev_bytes)
+{
+    if (!out || !dev_buf) return LCKV_EINVAL;
+    if (int rc = validate_config(cfg)) return rc;
+    if (reinterpret_cast<uintptr_t>(dev_buf) % 256) return LCKV_ENOMEM;
+    int sm = 0;
+    if (int rc = device_sm_count(&sm)) return rc;
+    lckv_cache* c = new (std::nothrow) lckv_cache();
+    if (!c) return LCKV_ENOMEM;
+    c->cfg = *cfg;
+    make_plan(cfg->n_layers, cfg->n_warmup, cfg->top_variant, c->plan);
+    c->n_kv_layers = 0;
+    for (int l = 0; l < cfg->n_layers; ++l) c->n_kv_layers += c->plan.write_slot[l] >= 0;
+    c->sm_count = sm;
+    c->grid = sm;
+    c->n_workers = sm * lckv::kAluWarps;
+    c->kernel_kind = resolve_kernel_kind(*cfg);
+    c->rows_per_tile = lckv::kAluSlotBytes / (cfg->head_dim * 2);
+    c->h_pairs = cfg->n_q_heads;
+    make_layout(*cfg, c->plan.n_slots, c->n_workers, c->n_kv_layers, c->lay);
+    if (dev_bytes < c->lay.total_bytes) { delete c; return LCKV_ENOMEM; }
+    const float scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale
+                                                 : 1.0f / std::sqrt((float)cfg->head_dim);
+    c->scale_log2 = scale * 1.4426950408889634f;
+    c->base = static_cast<uint8_t*>(dev_buf);
+    c->d_lens = reinterpret_cast<int32_t*>(c->base + c->lay.off_lens);
+    c->d_pre = reinterpret_cast<uint32_t*>(c->base + c->lay.off_pre);
+    c->d_start = reinterpret_cast<int32_t*>(c->base + c->lay.off_start);
+    c->d_counters = reinterpret_cast<int32_t*>(c->base + c->lay.off_counters);
+    c->d_status = reinterpret_cast<int32_t*>(c->base + c->lay.off_status);
+    c->d_partials = reinterpret_cast<float*>(c->base + c->lay.off_partials);
+    c->h_lens.assign(cfg->max_batch, 0);
+
+    bool ok = cuda_ok(cudaFuncSetAttribute(lckv::attn_alu_kernel<128>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           lckv::kAluSmemBytes)) &&
+              cuda_ok(cudaFuncSetAttribute(lckv::attn_alu_kernel<64>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           lckv::kAluSmemBytes)) &&
+              cuda_ok(cudaMemset(c->base, 0, c->lay.workspace_bytes)) &&
+              cuda_ok(cudaDeviceSynchronize());
+    if (!ok) { delete c; return LCKV_ECUDA; }
+    *out = c;
+    return LCKV_OK;
+}
+
+int lckv_cache_free(lckv_cache_t* cache)
+{
+    if (!cache) return LCKV_EINVAL;
+    delete cache;
+    return LCKV_OK;
+}
+
+int lckv_cache_info(const lckv_cache_t* c, lckv_info_t* info)
+{
+    if (!c || !info) return LCKV_EINVAL;
+    info->n_slots = c->plan.n_slots;
+    info->n_workers = c->n_workers;
+    info->rows_per_tile = c->rows_per_tile;
+    info->kernel_kind = c->kernel_kind;
+    int launches = 2 + c->cfg.n_layers + c->n_kv_layers;  // plan + advance + attention + appends
+    info->launches_per_step = launches;
+    info->sm_count = c->sm_count;
+    info->slot_bytes = c->lay.slot_bytes;
+    info->workspace_bytes = c->lay.workspace_bytes;
+    return LCKV_OK;
+}
+
+int lckv_cache_reset(lckv_cache_t* c, const int32_t* host_lens, int32_t batch, void* stream)
+{
+    if (!c || batch < 1 || batch > c->cfg.max_batch) return LCKV_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (host_lens) {
+        for (int b = 0; b < batch; ++b) {
+            if (host_lens[b] < 0) return LCKV_EINVAL;
+            if (host_lens[b] > c->cfg.max_seq) return LCKV_ECAPACITY;
+        }
+        for (int b = 0; b < batch; ++b) c->h_lens[b] = host_lens[b];
+        // h_lens is the staging source: it lives as long as the cache and pageable copies are
+        // staged before the call returns.
+        if (!cuda_ok(cudaMemcpyAsync(c->d_lens, c->h_lens.data(), (size_t)batch * 4,
+                                     cudaMemcpyHostToDevice, st)))
+            return LCKV_ECUDA;
+    } else {
+        for (int b = 0; b < batch; ++b) c->h_lens[b] = 0;
+        if (!cuda_ok(cudaMemsetAsync(c->d_lens, 0, (size_t)batch * 4, st))) return LCKV_ECUDA;
+    }
+    if (!cuda_ok(cudaMemsetAsync(c->d_counters, 0, (size_t)c->n_workers * 4, st))) return LCKV_ECUDA;
+    if (!cuda_ok(cudaMemsetAsync(c->d_status, 0, 4, st))) return LCKV_ECUDA;
+    return LCKV_OK;
+}
+
+int lckv_cache_lengths(const lckv_cache_t* c, int32_t* host_out, int32_t batch, void* stream)
+{
+    if (!c || !host_out || batch < 1 || batch > c->cfg.max_batch) return LCKV_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!cuda_ok(cudaMemcpyAsync(host_out, c->d_lens, (size_t)batch * 4, cudaMemcpyDeviceToHost, st)))
+        return LCKV_ECUDA;
+    return cuda_ok(cudaStreamSynchronize(st)) ? LCKV_OK : LCKV_ECUDA;
+}
+
+int lckv_cache_status(const lckv_cache_t* c, int32_t* host_status, void* stream)
+{
+    if (!c || !host_status) return LCKV_EINVAL;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (!cuda_ok(cudaMemcpyAsync(host_status, c->d_status, 4, cudaMemcpyDeviceToHost, st)))
+        return LCKV_ECUDA;
+    return cuda_ok(cudaStreamSynchronize(st)) ? LCKV_OK : LCKV_ECUDA;
+}
+
+int lckv_cache_slot_ptrs(const lckv_cache_t* c, int32_t slot, void** k, void** v)
+{
+    if (!c || !k || !v || slot < 0 || slot >= c->plan.n_slots) return LCKV_EINVAL;
+    *k = slot_k(c, slot);
+    *v = slot_v(c, slot);
+    return LCKV_OK;
+}
+
+int lckv_append_kv(lckv_cache_t* c, int32_t slot, const void* k_new, const void* v_new,
+                   int32_t batch, int32_t advance_len, void* stream)
+{
+    if (!c || !k_new || !v_new || batch < 1 || batch > c->cfg.max_batch) return LCKV_EINVAL;
+    if (slot < 0 || slot >= c->plan.n_slots) return LCKV_EINVAL;
+    if (max_len(c, batch) + 1 > c->cfg.max_seq) return LCKV_ECAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (int rc = launch_append(c, slot, k_new, v_new, batch, st)) return rc;
+    if (advance_len) return launch_advance(c, batch, st);
+    return LCKV_OK;
+}
+
+int lckv_decode_attention(lckv_cache_t* c, int32_t slot, int32_t mode, const void* q, void* out,
+                          float* lse, int32_t batch, void* stream)
+{
+    if (!c || !q || !out || batch < 1 || batch > c->cfg.max_batch) return LCKV_EINVAL;
+    if (slot < 0 || slot >= c->plan.n_slots) return LCKV_EINVAL;
+    if (mode != LCKV_MODE_CONDENSED && mode != LCKV_MODE_STANDARD) return LCKV_EINVAL;
+    if (max_len(c, batch) + mode > c->cfg.max_seq) return LCKV_ECAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (int rc = launch_plan(c, batch, st)) return rc;
+    return launch_attention(c, slot, mode, q, out, lse, batch, st);
+}
+
+int lckv_layer_stack_step(lckv_cache_t* c, const void* const* q_layers, void* const* out_layers,
+                          const void* const* k_new_layers, const void* const* v_new_layers,
+                          int32_t batch, void* stream)
+{
+    if (!c || !q_layers || !out_layers || !k_new_layers || !v_new_layers) return LCKV_EINVAL;
+    if (batch < 1 || batch > c->cfg.max_batch) return LCKV_EINVAL;
+    const int L = c->cfg.n_layers;
+    for (int l = 0; l < L; ++l) {
+        if (!q_layers[l] || !out_layers[l]) return LCKV_EINVAL;
+        if (c->plan.write_slot[l] >= 0 && (!k_new_layers[l] || !v_new_layers[l])) return LCKV_EINVAL;
+    }
+    if (max_len(c, batch) + 1 > c->cfg.max_seq) return LCKV_ECAPACITY;
+    return enqueue_step(c, q_layers, out_layers, k_new_layers, v_new_layers, batch,
+                        static_cast<cudaStream_t>(stream));
+}
+
+int lckv_layer_stack_step_host(lckv_cache_t* c, const void* const* q_host, void* const* out_host,
+                               const void* const* kn_host, const void* const* vn_host,
+                               int32_t batch, void* stream)
+{
+    if (!c || !q_host || !out_host || !kn_host || !vn_host) return LCKV_EINVAL;
+    if (!c->cfg.host_staging) return LCKV_EINVAL;
+    if (batch < 1 || batch > c->cfg.max_batch) return LCKV_EINVAL;
+    const int L = c->cfg.n_layers;
+    for (int l = 0; l < L; ++l) {
+        if (!q_host[l] || !out_host[l]) return LCKV_EINVAL;
+        if (c->plan.write_slot[l] >= 0 && (!kn_host[l] || !vn_host[l])) return LCKV_EINVAL;
+    }
+    if (max_len(c, batch) + 1 > c->cfg.max_seq) return LCKV_ECAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const size_t q_bytes = (size_t)batch * c->cfg.n_q_heads * c->cfg.head_dim * 2;
+    const size_t o_bytes = (size_t)batch * c->cfg.n_q_heads * c->cfg.head_dim * (c->cfg.out_dtype ? 4 : 2);
+    const size_t kv_bytes = (size_t)batch * c->cfg.n_kv_heads * c->cfg.head_dim * 2;
+    std::vector<const void*> dq(L), dk(L, nullptr), dv(L, nullptr);
+    std::vector<void*> dout(L);
+    int kv_i = 0;
+    for (int l = 0; l < L; ++l) {
+        uint8_t* sq = c->base + c->lay.off_stage_q + (size_t)l * c->lay.stage_q_bytes;
+        if (!cuda_ok(cudaMemcpyAsync(sq, q_host[l], q_bytes, cudaMemcpyHostToDevice, st)))
+            return LCKV_ECUDA;
+        dq[l] = sq;
+        dout[l] = c->base + c->lay.off_stage_out + (size_t)l * c->lay.stage_out_bytes;
+        if (c->plan.write_slot[l] >= 0) {
+            uint8_t* sk = c->base + c->lay.off_stage_kv + (size_t)(2 * kv_i) * c->lay.stage_kv_bytes;
+            uint8_t* sv = sk + c->lay.stage_kv_bytes;
+            if (!cuda_ok(cudaMemcpyAsync(sk, kn_host[l], kv_bytes, cudaMemcpyHostToDevice, st)) ||
+                !cuda_ok(cudaMemcpyAsync(sv, vn_host[l], kv_bytes, cudaMemcpyHostToDevice, st)))
+                return LCKV_ECUDA;
+            dk[l] = sk;
+            dv[l] = sv;
+            ++kv_i;
+        }
+    }
+    if (int rc = enqueue_step(c, dq.data(), dout.data(), dk.data(), dv.data(), batch, st)) return rc;
+    for (int l = 0; l < L; ++l)
+        if (!cuda_ok(cudaMemcpyAsync(out_host[l], dout[l], o_bytes, cudaMemcpyDeviceToHost, st)))
+            return LCKV_ECUDA;
+    return LCKV_OK;
+}
+
+const char* lckv_status_string(int s)
+{
+    switch (s) {
+        case LCKV_OK: return "ok";
+        case LCKV_EINVAL: return "invalid argument";
+        case LCKV_ECAPACITY: return "sequence capacity exceeded";
+        case LCKV_ENOMEM: return "device buffer too small or misaligned";
+        case LCKV_ECUDA: return "CUDA call failed";
+        case LCKV_ETIMEOUT: return "device-side wait timed out";
+        default: return "unknown status";
+    }
+}
+
+int lckv_last_cuda_error(void) { return g_last_cuda_error; }
+
+}  // extern "C"

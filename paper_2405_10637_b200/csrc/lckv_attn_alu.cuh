@@ -1,0 +1,385 @@
+// Decode attention, FP32-ALU kernel: one query head per (sequence, head) pair.
+//
+// This is the kernel for multi-head attention (group size 1, 1 flop per KV byte): the work is
+// streaming K and V rows from HBM, so it is organised around keeping many bulk copies in flight.
+//
+//  * A launch is one long sequence of tiles (R cache rows of one (b, head) pair; see plan_kernel),
+//    cut into equal contiguous ranges, one per WORKER.  A worker is one warp: it owns a private
+//    ring of shared-memory slots, issues its own 1-D bulk (TMA) copies K-tile, V-tile, K-tile, ...
+//    into the ring (lane 0), waits on the slot's mbarrier, and consumes the rows with plain FP32
+//    FMAs.  No block-level synchronisation exists after start-up.
+//  * Softmax is the running-max form (fp32, base-2 exponentials); the state (m, l, o[D]) lives in
+//    registers across the tiles of a pair.
+//  * A pair that falls entirely inside one worker's range is normalised and written directly.
+//    A pair cut by a range boundary leaves an fp32 partial (m, l, o) per contributing worker; the
+//    contributor that arrives last (atomic ticket, no waiting) merges them with the log-sum-exp
+//    rule in a fixed order and writes the row.
+#pragma once
+#include "lckv_device.cuh"
+
+namespace lckv {
+
+constexpr int kAluWarps = 8;         // workers per CTA
+constexpr int kAluSlots = 6;         // ring slots per worker
+constexpr int kAluSlotBytes = 4096;  // one tile of K or of V
+constexpr int kAluSmemBytes = kAluWarps * kAluSlots * (kAluSlotBytes + 8);
+
+struct AttnParams {
+    const uint16_t* K;        // [B_max, H_kv, T_cap, D] bf16
+    const uint16_t* V;
+    const uint16_t* q;        // [B, H_q, D] bf16
+    void* out;                // [B, H_q, D] bf16 or fp32
+    float* lse;               // [B, H_q] or null
+    const int32_t* lens;      // [B]
+    const uint32_t* pre;      // [B + 1] tile prefix for this mode
+    const int32_t* start_b;   // [n_workers] for this mode
+    float* partials;          // [2 * n_workers][D + 4]
+    int32_t* counters;        // [n_workers], zero between launches
+    int32_t* status;          // device status word
+    int64_t T_cap;
+    int32_t B, H_q, H_kv, mode, n_workers, out_f32;
+    float scale_log2;         // softmax scale * log2(e)
+};
+
+struct TileCursor {
+    int32_t b, h;
+    uint32_t t, nt;   // tile within the pair; tiles per pair of sequence b
+    int32_t nv;       // visible rows of sequence b
+};
+
+__device__ __forceinline__ void cursor_load(TileCursor& c, const AttnParams& p)
+{
+    c.nt = __ldg(p.pre + c.b + 1) - __ldg(p.pre + c.b);
+    c.nv = __ldg(p.lens + c.b) + p.mode;
+}
+
+// Next tile in (b, pair, tile) order, skipping sequences without tiles.  Safe past the end.
+__device__ __forceinline__ void cursor_next(TileCursor& c, const AttnParams& p, int H)
+{
+    if (++c.t < c.nt) return;
+    c.t = 0;
+    if (++c.h < H) return;
+    c.h = 0;
+    do {
+        if (++c.b >= p.B) { c.b = p.B; c.nt = 0; c.nv = 0; return; }
+        cursor_load(c, p);
+    } while (c.nt == 0);
+}
+
+template <int D>
+__global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnParams p)
+{
+    constexpr int R = kAluSlotBytes / (D * 2);  // rows per tile: 16 (D=128), 32 (D=64)
+    constexpr int LPR = D / 8;                  // lanes per row (16 bytes each)
+    constexpr int RPI = 32 / LPR;               // rows covered by one warp-wide 16-byte load
+    constexpr int NP = R / RPI;                 // such loads per tile = partial sums per lane
+    constexpr int DUP = LPR / NP;               // lanes that end up holding the same score
+    constexpr int NS = kAluSlots;
+    constexpr int REC = D + 4;                  // floats per partial record
+    static_assert(NP == 8 && (DUP == 1 || DUP == 2), "layout assumes 8 partial sums per lane");
+
+    extern __shared__ __align__(128) uint8_t smem[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int w = blockIdx.x * kAluWarps + warp;
+    const int H = p.H_q;
+    const int g = p.H_q / p.H_kv;
+    const uint32_t FULL = 0xffffffffu;
+
+    const uint32_t ring = smem_u32(smem) + warp * (NS * kAluSlotBytes);
+    const uint32_t bars = smem_u32(smem) + kAluWarps * NS * kAluSlotBytes + warp * (NS * 8);
+    if (lane == 0) {
+        for (int s = 0; s < NS; ++s) mbar_init(bars + 8 * s, 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+
+    // Rows that see nothing (diagonal-masked first token): the zero dummy KV gives o = 0, lse = 0.
+    for (int b = w; b < p.B; b += p.n_workers) {
+        if (__ldg(p.lens + b) + p.mode == 0) {
+            const int esz = p.out_f32 ? 4 : 2;
+            const int n16 = H * D * esz / 16;
+            uint4* o16 = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.out) +
+                                                  (size_t)b * H * D * esz);
+            for (int i = lane; i < n16; i += 32) o16[i] = make_uint4(0, 0, 0, 0);
+            if (p.lse)
+                for (int i = lane; i < H; i += 32) p.lse[(size_t)b * H + i] = 0.f;
+        }
+    }
+
+    const uint64_t total = (uint64_t)__ldg(p.pre + p.B) * (uint64_t)H;
+    if (total == 0) return;
+    const uint64_t n_eff = total < (uint64_t)p.n_workers ? total : (uint64_t)p.n_workers;
+    if ((uint64_t)w >= n_eff) return;
+    const uint64_t lo = (uint64_t)w * total / n_eff;
+    const uint64_t hi = (uint64_t)(w + 1) * total / n_eff;
+    const uint32_t n_tiles = (uint32_t)(hi - lo);
+    const uint32_t n_items = 2 * n_tiles;
+
+    TileCursor cc;
+    cc.b = __ldg(p.start_b + w);
+    cursor_load(cc, p);
+    {
+        const uint64_t rel = lo - (uint64_t)__ldg(p.pre + cc.b) * (uint64_t)H;
+        cc.h = (int32_t)(rel / cc.nt);
+        cc.t = (uint32_t)(rel % cc.nt);
+    }
+    TileCursor ci = cc;
+
+    uint32_t issued = 0, islot = 0;
+    auto issue = [&]() {
+        const int rows = min(R, ci.nv - (int)ci.t * R);
+        const uint32_t bytes = (uint32_t)rows * (D * 2);
+        const uint16_t* base = (issued & 1) ? p.V : p.K;
+        const uint16_t* src =
+            base + (((int64_t)ci.b * p.H_kv + ci.h / g) * p.T_cap + (int64_t)ci.t * R) * D;
+        if (lane == 0) {
+            mbar_expect_tx(bars + 8 * islot, bytes);
+            bulk_g2s(ring + islot * kAluSlotBytes, src, bytes, bars + 8 * islot);
+        }
+        if (issued & 1) cursor_next(ci, p, H);
+        ++issued;
+        islot = (islot + 1 == NS) ? 0 : islot + 1;
+    };
+    {
+        const uint32_t pro = n_items < (uint32_t)NS ? n_items : (uint32_t)NS;
+        while (issued < pro) issue();
+    }
+
+    const int grp = lane / LPR;  // which of the RPI rows of a load this lane reads
+    const int a = lane % LPR;    // which 16 bytes of the row
+    uint32_t cslot = 0, cphase = 0;
+    bool ok = true;
+
+    float qf[8];
+    auto load_q = [&](const TileCursor& c) {
+        const uint4 raw =
+            __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)c.b * H + c.h) * D) + a);
+        qf[0] = bf16lo(raw.x) * p.scale_log2; qf[1] = bf16hi(raw.x) * p.scale_log2;
+        qf[2] = bf16lo(raw.y) * p.scale_log2; qf[3] = bf16hi(raw.y) * p.scale_log2;
+        qf[4] = bf16lo(raw.z) * p.scale_log2; qf[5] = bf16hi(raw.z) * p.scale_log2;
+        qf[6] = bf16lo(raw.w) * p.scale_log2; qf[7] = bf16hi(raw.w) * p.scale_log2;
+    };
+    load_q(cc);
+    uint32_t seg_t0 = cc.t;
+    float m_run = -INFINITY, l_run = 0.f;
+    float o[8];
+#pragma unroll
+    for (int k = 0; k < 8; ++k) o[k] = 0.f;
+
+    for (uint32_t tile = 0; tile < n_tiles; ++tile) {
+        const int rows = min(R, cc.nv - (int)cc.t * R);
+
+        // ---- K tile: scores -----------------------------------------------------------------
+        if (!mbar_wait_bounded(bars + 8 * cslot, cphase)) { ok = false; break; }
+        float part[NP];
+        {
+            const uint32_t base = ring + cslot * kAluSlotBytes + grp * (D * 2) + a * 16;
+#pragma unroll
+            for (int i = 0; i < NP; ++i) {
+                const uint4 kv = lds128(base + i * (RPI * D * 2));
+                float s = bf16lo(kv.x) * qf[0];
+                s = fmaf(bf16hi(kv.x), qf[1], s);
+                s = fmaf(bf16lo(kv.y), qf[2], s);
+                s = fmaf(bf16hi(kv.y), qf[3], s);
+                s = fmaf(bf16lo(kv.z), qf[4], s);
+                s = fmaf(bf16hi(kv.z), qf[5], s);
+                s = fmaf(bf16lo(kv.w), qf[6], s);
+                s = fmaf(bf16hi(kv.w), qf[7], s);
+                part[i] = s;
+            }
+        }
+        __syncwarp();
+        if (issued < n_items) issue();  // refill the slot just read
+        cslot = (cslot + 1 == NS) ? 0 : cslot + 1;
+        if (cslot == 0) cphase ^= 1;
+
+        // Sum each row's LPR partial dot products.  Exchange steps halve the number of values a
+        // lane carries (8 -> 4 -> 2 -> 1); with 16 lanes per row one plain butterfly step remains.
+        {
+            bool up = (a & (LPR / 2)) != 0;
+#pragma unroll
+            for (int k = 0; k < 4; ++k) {
+                const float send = up ? part[k] : part[k + 4];
+                const float keep = up ? part[k + 4] : part[k];
+                part[k] = keep + __shfl_xor_sync(FULL, send, LPR / 2);
+            }
+            up = (a & (LPR / 4)) != 0;
+#pragma unroll
+            for (int k = 0; k < 2; ++k) {
+                const float send = up ? part[k] : part[k + 2];
+                const float keep = up ? part[k + 2] : part[k];
+                part[k] = keep + __shfl_xor_sync(FULL, send, LPR / 4);
+            }
+            up = (a & (LPR / 8)) != 0;
+            {
+                const float send = up ? part[0] : part[1];
+                const float keep = up ? part[1] : part[0];
+                part[0] = keep + __shfl_xor_sync(FULL, send, LPR / 8);
+            }
+            if (DUP == 2) part[0] += __shfl_xor_sync(FULL, part[0], 1);
+        }
+        // This lane now holds the score of load index a / DUP, i.e. of tile row:
+        const int my_row = (a / DUP) * RPI + grp;
+        const float s = (my_row < rows) ? part[0] : -INFINITY;
+
+        float m_tile = s;
+#pragma unroll
+        for (int off = 16; off >= 1; off >>= 1)
+            m_tile = fmaxf(m_tile, __shfl_xor_sync(FULL, m_tile, off));
+        const float m_new = fmaxf(m_run, m_tile);
+        const float alpha = ex2(m_run - m_new);
+        const float pr = ex2(s - m_new);
+        l_run = fmaf(l_run, alpha, pr);
+        m_run = m_new;
+#pragma unroll
+        for (int k = 0; k < 8; ++k) o[k] *= alpha;
+
+        // ---- V tile: weighted sum -----------------------------------------------------------
+        if (!mbar_wait_bounded(bars + 8 * cslot, cphase)) { ok = false; break; }
+        if (rows < R) {
+            // Rows past the copy hold leftovers of an earlier tile; their weight is 0 but 0 * NaN
+            // is NaN, so clear them.  Generic-proxy writes, fenced before the slot's next copy.
+            const uint32_t vb = ring + cslot * kAluSlotBytes;
+            for (int i = rows * (D * 2) + lane * 16; i < R * D * 2; i += 32 * 16)
+                sts128(vb + i, make_uint4(0, 0, 0, 0));
+            fence_proxy_async_smem();
+            __syncwarp();
+        }
+        {
+            const uint32_t base = ring + cslot * kAluSlotBytes + grp * (D * 2) + a * 16;
+#pragma unroll
+            for (int i = 0; i < NP; ++i) {
+                const float pi = __shfl_sync(FULL, pr, grp * LPR + i * DUP);
+                const uint4 vv = lds128(base + i * (RPI * D * 2));
+                o[0] = fmaf(pi, bf16lo(vv.x), o[0]);
+                o[1] = fmaf(pi, bf16hi(vv.x), o[1]);
+                o[2] = fmaf(pi, bf16lo(vv.y), o[2]);
+                o[3] = fmaf(pi, bf16hi(vv.y), o[3]);
+                o[4] = fmaf(pi, bf16lo(vv.z), o[4]);
+                o[5] = fmaf(pi, bf16hi(vv.z), o[5]);
+                o[6] = fmaf(pi, bf16lo(vv.w), o[6]);
+                o[7] = fmaf(pi, bf16hi(vv.w), o[7]);
+            }
+        }
+        __syncwarp();
+        if (issued < n_items) issue();
+        cslot = (cslot + 1 == NS) ? 0 : cslot + 1;
+        if (cslot == 0) cphase ^= 1;
+
+        // ---- end of this worker's part of the pair? -----------------------------------------
+        const bool pair_end = (cc.t + 1 == cc.nt);
+        const bool last = (tile + 1 == n_tiles);
+        if (pair_end || last) {
+            // everything this worker saw of the pair: reduce over row groups and lanes
+#pragma unroll
+            for (int off = LPR; off < 32; off <<= 1)
+#pragma unroll
+                for (int k = 0; k < 8; ++k) o[k] += __shfl_xor_sync(FULL, o[k], off);
+            float l_tot = l_run;
+#pragma unroll
+            for (int off = 16; off >= 1; off >>= 1) l_tot += __shfl_xor_sync(FULL, l_tot, off);
+            l_tot *= (1.0f / DUP);
+            float m_fin = m_run;
+
+            const bool complete = pair_end && seg_t0 == 0;
+            bool write_row = complete;
+            if (!complete) {
+                const uint64_t gs = (uint64_t)__ldg(p.pre + cc.b) * (uint64_t)H +
+                                    (uint64_t)cc.h * cc.nt;  // the pair's first global tile
+                const uint64_t ge = gs + cc.nt;
+                const uint32_t c_first = (uint32_t)(((gs + 1) * n_eff - 1) / total);
+                const uint32_t c_last = (uint32_t)((ge * n_eff - 1) / total);
+                const bool at_lo = (gs + seg_t0 == lo);
+                float* rec = p.partials + (size_t)(2 * w + (at_lo ? 0 : 1)) * REC;
+                if (lane < LPR) {
+                    reinterpret_cast<float4*>(rec)[2 * lane] = make_float4(o[0], o[1], o[2], o[3]);
+                    reinterpret_cast<float4*>(rec)[2 * lane + 1] =
+                        make_float4(o[4], o[5], o[6], o[7]);
+                }
+                if (lane == 0) { rec[D] = m_fin; rec[D + 1] = l_tot; }
+                __threadfence();
+                __syncwarp();
+                int ticket = 0;
+                if (lane == 0) ticket = atomicAdd(p.counters + c_first, 1);
+                ticket = __shfl_sync(FULL, ticket, 0);
+                if (ticket == (int)(c_last - c_first)) {
+                    // Last contributor: merge every part in worker order (fixed summation order).
+                    __threadfence();
+                    float M = -INFINITY;
+                    for (uint32_t c = c_first; c <= c_last; ++c) {
+                        const uint64_t lo_c = (uint64_t)c * total / n_eff;
+                        const float* r = p.partials +
+                            (size_t)(2 * c + ((c == c_first && gs != lo_c) ? 1 : 0)) * REC;
+                        M = fmaxf(M, __ldcg(r + D));
+                    }
+                    float Lsum = 0.f, acc[8];
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+                    for (uint32_t c = c_first; c <= c_last; ++c) {
+                        const uint64_t lo_c = (uint64_t)c * total / n_eff;
+                        const float* r = p.partials +
+                            (size_t)(2 * c + ((c == c_first && gs != lo_c) ? 1 : 0)) * REC;
+                        const float wgt = ex2(__ldcg(r + D) - M);
+                        Lsum = fmaf(__ldcg(r + D + 1), wgt, Lsum);
+                        if (lane < LPR) {
+                            const float4 x0 = __ldcg(reinterpret_cast<const float4*>(r) + 2 * lane);
+                            const float4 x1 =
+                                __ldcg(reinterpret_cast<const float4*>(r) + 2 * lane + 1);
+                            acc[0] = fmaf(x0.x, wgt, acc[0]); acc[1] = fmaf(x0.y, wgt, acc[1]);
+                            acc[2] = fmaf(x0.z, wgt, acc[2]); acc[3] = fmaf(x0.w, wgt, acc[3]);
+                            acc[4] = fmaf(x1.x, wgt, acc[4]); acc[5] = fmaf(x1.y, wgt, acc[5]);
+                            acc[6] = fmaf(x1.z, wgt, acc[6]); acc[7] = fmaf(x1.w, wgt, acc[7]);
+                        }
+                    }
+#pragma unroll
+                    for (int k = 0; k < 8; ++k) o[k] = acc[k];
+                    l_tot = Lsum;
+                    m_fin = M;
+                    write_row = true;
+                    if (lane == 0) p.counters[c_first] = 0;  // ready for the next launch
+                }
+            }
+            if (write_row) {
+                const float inv = 1.0f / l_tot;
+                const size_t row = (size_t)cc.b * H + cc.h;
+                if (lane < LPR) {
+                    if (p.out_f32) {
+                        float4* dst =
+                            reinterpret_cast<float4*>(static_cast<float*>(p.out) + row * D);
+                        dst[2 * lane] = make_float4(o[0] * inv, o[1] * inv, o[2] * inv, o[3] * inv);
+                        dst[2 * lane + 1] =
+                            make_float4(o[4] * inv, o[5] * inv, o[6] * inv, o[7] * inv);
+                    } else {
+                        uint4 pk;
+                        pk.x = pack_bf16x2(o[0] * inv, o[1] * inv);
+                        pk.y = pack_bf16x2(o[2] * inv, o[3] * inv);
+                        pk.z = pack_bf16x2(o[4] * inv, o[5] * inv);
+                        pk.w = pack_bf16x2(o[6] * inv, o[7] * inv);
+                        reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + row * D)[lane] = pk;
+                    }
+                }
+                if (p.lse && lane == 0) p.lse[row] = (m_fin + lg2(l_tot)) * 0.6931471805599453f;
+            }
+            m_run = -INFINITY;
+            l_run = 0.f;
+#pragma unroll
+            for (int k = 0; k < 8; ++k) o[k] = 0.f;
+        }
+        if (!last) {
+            cursor_next(cc, p, H);
+            if (pair_end) { load_q(cc); seg_t0 = 0; }
+        }
+    }
+
+    if (!ok) {
+        // A copy never landed.  Report it, give the copies still in flight a bounded chance to
+        // finish (they target this CTA's shared memory), and leave.
+        if (lane == 0) atomicExch(p.status, kStatusTimeout);
+        for (int s = 0; s < NS; ++s) {
+            mbar_wait_bounded(bars + 8 * s, 0, 1u << 10);
+            mbar_wait_bounded(bars + 8 * s, 1, 1u << 10);
+        }
+    }
+}
+
+}  // namespace lckv

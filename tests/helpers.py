@@ -1,0 +1,111 @@
+"""Shared machinery of the GPU parity tests: build a cache, fill it, step it, compare with the oracle."""
+import numpy as np
+import torch
+
+from oracle import lckv_oracle as orc
+from paper_2405_10637_b200 import binding as lk
+from paper_2405_10637_b200 import inputs as syn
+
+MAX_ABS = 1e-2     # tolerance on |gpu - oracle| per element
+REL_L2 = 5e-3      # tolerance on ||gpu - oracle||_2 / ||oracle||_2
+NAN_BITS = 0x7FC0  # bf16 quiet NaN, used to poison rows that must never be read
+
+
+def compare(got, want, what=""):
+    """got: torch tensor (bf16/fp32) from the GPU; want: float64 numpy from the oracle."""
+    g = got.detach().float().cpu().numpy().astype(np.float64)
+    assert g.shape == want.shape, (g.shape, want.shape)
+    assert np.isfinite(g).all(), f"{what}: non-finite GPU output"
+    zero_rows = ~want.any(axis=-1)
+    assert not g[zero_rows].any(), f"{what}: rows the oracle gives as exactly 0 are not 0"
+    max_abs = np.abs(g - want).max() if g.size else 0.0
+    denom = np.linalg.norm(want[~zero_rows])
+    rel = np.linalg.norm((g - want)[~zero_rows]) / denom if denom > 0 else 0.0
+    assert max_abs <= MAX_ABS, f"{what}: max-abs {max_abs:.3e}"
+    assert rel <= REL_L2, f"{what}: rel-L2 {rel:.3e}"
+    return max_abs, rel
+
+
+class Case:
+    """One layer stack with GPU cache and host (oracle) caches holding the same bits."""
+
+    def __init__(self, L, w, Hq, Hkv, d, lens, T_cap, variant=0, out_dtype=0, seed=1234, std=1.0,
+                 poison=True, B_max=None, scale=0.0, kernel_kind=0, host_staging=0, use_graph=0):
+        self.L, self.w, self.Hq, self.Hkv, self.d = L, w, Hq, Hkv, d
+        self.lens = np.asarray(lens, np.int32).copy()
+        self.B = len(lens)
+        self.T_cap, self.variant, self.seed, self.std = T_cap, variant, seed, std
+        B_max = B_max or self.B
+        self.cfg = lk.make_config(L, w, Hq, Hkv, d, B_max, T_cap, softmax_scale=scale,
+                                  top_variant=variant, out_dtype=out_dtype, kernel_kind=kernel_kind,
+                                  host_staging=host_staging, use_graph=use_graph)
+        self.scale = scale if scale > 0 else d ** -0.5
+        self.cache = lk.Cache(self.cfg)
+        self.plan = orc.plan(L, w, variant)
+        self.n_slots = self.plan["n_slots"]
+        assert self.cache.info.n_slots == self.n_slots
+        self.hK, self.hV = [], []
+        for s in range(self.n_slots):
+            kb = syn.bits(syn.randn_bf16((B_max, Hkv, T_cap, d), seed + 2 * s, std=std))
+            vb = syn.bits(syn.randn_bf16((B_max, Hkv, T_cap, d), seed + 2 * s + 1, std=std))
+            if poison:
+                for b in range(B_max):
+                    n = int(self.lens[b]) if b < self.B else 0
+                    kb[b, :, n:] = NAN_BITS
+                    vb[b, :, n:] = NAN_BITS
+            kt, vt = self.cache.slot_tensors(s)
+            kt.copy_(syn.from_bits(kb)); vt.copy_(syn.from_bits(vb))
+            self.hK.append(kb); self.hV.append(vb)
+        self.cache.lckv_cache_reset(self.lens.tolist())
+        self.step_no = 0
+
+    def step_inputs(self):
+        s0 = self.seed + 1000 * (self.step_no + 1)
+        q = [syn.randn_bf16((self.B, self.Hq, self.d), s0 + l, std=self.std) for l in range(self.L)]
+        kn = [syn.randn_bf16((self.B, self.Hkv, self.d), s0 + 200 + l, std=self.std)
+              if self.plan["write_slot"][l] >= 0 else None for l in range(self.L)]
+        vn = [syn.randn_bf16((self.B, self.Hkv, self.d), s0 + 400 + l, std=self.std)
+              if self.plan["write_slot"][l] >= 0 else None for l in range(self.L)]
+        return q, kn, vn
+
+    def step(self, check=True, host=False):
+        q, kn, vn = self.step_inputs()
+        odt = torch.float32 if self.cfg.out_dtype else torch.bfloat16
+        if host:
+            qd = [t.pin_memory() for t in q]
+            knd = [None if t is None else t.pin_memory() for t in kn]
+            vnd = [None if t is None else t.pin_memory() for t in vn]
+            outs = [torch.empty((self.B, self.Hq, self.d), dtype=odt).pin_memory() for _ in range(self.L)]
+            self.cache.lckv_layer_stack_step_host(qd, outs, knd, vnd)
+        else:
+            dev = self.cache.device
+            qd = [t.to(dev) for t in q]
+            knd = [None if t is None else t.to(dev) for t in kn]
+            vnd = [None if t is None else t.to(dev) for t in vn]
+            outs = [torch.full((self.B, self.Hq, self.d), float("nan"), dtype=odt, device=dev)
+                    for _ in range(self.L)]
+            self.cache.lckv_layer_stack_step(qd, outs, knd, vnd)
+        torch.cuda.synchronize()
+        assert self.cache.lckv_cache_status() == 0
+        want, _ = orc.stack_step(self.L, self.w, [syn.bits(t) for t in q],
+                                 [None if t is None else syn.bits(t) for t in kn],
+                                 [None if t is None else syn.bits(t) for t in vn],
+                                 self.hK, self.hV, self.lens, self.scale, top_variant=self.variant)
+        self.step_no += 1
+        stats = []
+        if check:
+            for l in range(self.L):
+                stats.append(compare(outs[l], want[l], f"layer {l} step {self.step_no}"))
+            self.check_state()
+        return outs, want, stats
+
+    def check_state(self):
+        """Lengths and every byte of every cache, bit for bit."""
+        assert self.cache.lckv_cache_lengths(self.B) == self.lens.tolist()
+        for s in range(self.n_slots):
+            kt, vt = self.cache.slot_tensors(s)
+            assert np.array_equal(syn.bits(kt), self.hK[s]), f"slot {s} K differs"
+            assert np.array_equal(syn.bits(vt), self.hV[s]), f"slot {s} V differs"
+
+    def close(self):
+        self.cache.close()

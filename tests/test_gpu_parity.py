@@ -1,0 +1,176 @@
+"""GPU parity: the CUDA library (through its C ABI) against the float64 oracle, element by element
+on the same seeded bf16 inputs.  Tolerances: max-abs 1e-2, relative L2 5e-3 (bf16 inputs and
+outputs, fp32 arithmetic); lengths, append positions and every cache byte bit-exact."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lckv_oracle as orc
+from paper_2405_10637_b200 import binding as lk
+from paper_2405_10637_b200 import inputs as syn
+from helpers import Case, compare, NAN_BITS
+
+pytestmark = pytest.mark.gpu
+
+
+def test_toy_config_w0_all_layers_read_shared_cache():
+    """4 layers, MHA 4 heads, d_h 64, w = 0, batch 2, 128 cached tokens, everything from seed 0 in
+    the order K, V, q, k_new, v_new."""
+    L, H, d, B, T = 4, 4, 64, 2, 128
+    K, V, *rest = syn.draw_sequence([(B, H, T + 1, d)] * 2 + [(B, H, d)] * L + [(B, H, d)] * 2, 0)
+    q, (kn, vn) = rest[:L], rest[L:]
+    cfg = lk.make_config(L, 0, H, H, d, B, T + 1)
+    cache = lk.Cache(cfg)
+    kt, vt = cache.slot_tensors(0)
+    kt.copy_(K); vt.copy_(V)
+    cache.lckv_cache_reset([T] * B)
+    dev = cache.device
+    outs = [torch.empty((B, H, d), dtype=torch.bfloat16, device=dev) for _ in range(L)]
+    cache.lckv_layer_stack_step([t.to(dev) for t in q], outs, [None] * (L - 1) + [kn.to(dev)],
+                                [None] * (L - 1) + [vn.to(dev)])
+    torch.cuda.synchronize()
+    hK, hV = syn.bits(K), syn.bits(V)
+    lens = np.full(B, T, np.int32)
+    want, _ = orc.stack_step(L, 0, [syn.bits(t) for t in q], [None] * (L - 1) + [syn.bits(kn)],
+                             [None] * (L - 1) + [syn.bits(vn)], [hK], [hV], lens, d ** -0.5)
+    for l in range(L):
+        compare(outs[l], want[l], f"layer {l}")
+    assert cache.lckv_cache_lengths(B) == [T + 1] * B
+    kt, vt = cache.slot_tensors(0)
+    assert np.array_equal(syn.bits(kt), hK) and np.array_equal(syn.bits(vt), hV)
+    cache.close()
+
+
+@pytest.mark.parametrize("d", [64, 128])
+@pytest.mark.parametrize("variant", [0, 1])
+def test_small_ragged_stack_with_edge_lengths(d, variant):
+    """Lengths around the tile edges (0, 1, R-1, R, R+1, ...), T_cap not a multiple of the tile,
+    NaN poison beyond every length, w = 2 sandwich, three consecutive steps."""
+    lens = [0, 1, 15, 16, 17, 31, 32, 33, 63, 64, 65, 100, 257, 300]
+    c = Case(L=5, w=2, Hq=4, Hkv=4, d=d, lens=lens, T_cap=303, variant=variant, seed=77 + d)
+    for _ in range(3):
+        c.step()
+    c.close()
+
+
+@pytest.mark.parametrize("w", [0, 2, 4])
+def test_many_pairs_per_worker(w):
+    """More tiles than workers: whole (sequence, head) pairs inside one worker's range are written
+    directly, pairs cut by a range boundary go through the partial merge."""
+    lens = syn.ragged_lengths(96, 40, 400, 5).tolist()
+    c = Case(L=4, w=w, Hq=16, Hkv=16, d=128, lens=lens, T_cap=402, seed=900 + w)
+    c.step(); c.step()
+    c.close()
+
+
+def test_w_equals_L_standard_transformer():
+    c = Case(L=3, w=3, Hq=8, Hkv=8, d=128, lens=[5, 0, 77, 130], T_cap=140, seed=31)
+    c.step(); c.step()
+    c.close()
+
+
+def test_gqa_group_of_8_and_of_2():
+    """Grouped heads: q head h reads kv head h // g."""
+    c = Case(L=4, w=2, Hq=32, Hkv=4, d=64, lens=[3, 64, 200, 511], T_cap=520, seed=8, std=0.125)
+    c.step(); c.step()
+    c.close()
+    c = Case(L=3, w=0, Hq=8, Hkv=4, d=128, lens=[1, 90, 33], T_cap=100, seed=9)
+    c.step()
+    c.close()
+
+
+def test_fp32_outputs_are_tight():
+    """With fp32 outputs only the arithmetic differs: errors two orders below the bf16 bound."""
+    c = Case(L=3, w=2, Hq=8, Hkv=8, d=128, lens=[9, 500, 1000, 17], T_cap=1024, out_dtype=1, seed=5)
+    _, _, stats = c.step()
+    assert max(s[0] for s in stats) < 2e-5 and max(s[1] for s in stats) < 2e-5
+    c.close()
+
+
+def test_single_long_sequence_split_over_many_workers():
+    """One sequence, one head: every worker holds a slice of the same pair (deepest merge)."""
+    c = Case(L=2, w=0, Hq=1, Hkv=1, d=128, lens=[40000], T_cap=40010, seed=3, out_dtype=1)
+    c.step()
+    c.close()
+
+
+def test_decode_attention_entry_lse_and_single_key_exactness():
+    """Per-layer entry point: log-sum-exp output; one visible key gives o = v_0 bit-exactly."""
+    B, H, d, T = 3, 4, 128, 50
+    cfg = lk.make_config(2, 0, H, H, d, B, T)
+    cache = lk.Cache(cfg)
+    K = syn.randn_bf16((B, H, T, d), 1); V = syn.randn_bf16((B, H, T, d), 2)
+    kt, vt = cache.slot_tensors(0); kt.copy_(K); vt.copy_(V)
+    lens = [1, 0, 37]
+    cache.lckv_cache_reset(lens)
+    q = syn.randn_bf16((B, H, d), 3)
+    lse = torch.full((B, H), float("nan"), device=cache.device)
+    out = cache.lckv_decode_attention(0, lk.MODE_CONDENSED, q.to(cache.device), lse=lse)
+    torch.cuda.synchronize()
+    want, want_lse = orc.decode_attention(syn.bits(q), syn.bits(K), syn.bits(V),
+                                          np.array(lens, np.int32), 0, d ** -0.5)
+    compare(out, want)
+    np.testing.assert_allclose(lse.cpu().numpy(), want_lse, atol=2e-3)
+    assert np.array_equal(syn.bits(out[0]), syn.bits(V[0, :, 0]))      # len 1: o = v_0 exactly
+    assert not out[1].float().abs().sum().item() and not lse[1].abs().sum().item()  # len 0
+    # standard mode needs row len appended first (without advancing)
+    kn = syn.randn_bf16((B, H, d), 4); vn = syn.randn_bf16((B, H, d), 5)
+    cache.lckv_append_kv(0, kn.to(cache.device), vn.to(cache.device), advance_len=0)
+    out1 = cache.lckv_decode_attention(0, lk.MODE_STANDARD, q.to(cache.device))
+    hK, hV = syn.bits(K), syn.bits(V)
+    orc.append(hK, hV, syn.bits(kn), syn.bits(vn), np.array(lens, np.int32))
+    want1, _ = orc.decode_attention(syn.bits(q), hK, hV, np.array(lens, np.int32), 1, d ** -0.5)
+    compare(out1, want1)
+    assert cache.lckv_cache_lengths(B) == lens
+    cache.close()
+
+
+def test_errors_capacity_and_arguments():
+    B, H, d, T = 2, 2, 64, 8
+    cfg = lk.make_config(2, 0, H, H, d, B, T)
+    cache = lk.Cache(cfg)
+    cache.lckv_cache_reset([8, 3])          # sequence 0 is full
+    dev = cache.device
+    q = torch.zeros((B, H, d), dtype=torch.bfloat16, device=dev)
+    kt0 = syn.bits(cache.slot_tensors(0)[0]).copy()
+    with pytest.raises(lk.LckvError) as e:
+        cache.lckv_layer_stack_step([q, q], [q.clone(), q.clone()], [None, q], [None, q])
+    assert e.value.status == lk.ECAPACITY
+    with pytest.raises(lk.LckvError) as e:
+        cache.lckv_append_kv(0, q, q)
+    assert e.value.status == lk.ECAPACITY
+    assert cache.lckv_cache_lengths(B) == [8, 3]
+    assert np.array_equal(syn.bits(cache.slot_tensors(0)[0]), kt0)
+    cache.lckv_decode_attention(0, lk.MODE_CONDENSED, q)   # reading a full cache is fine
+    for bad in [dict(slot=1, mode=0), dict(slot=0, mode=2), dict(slot=-1, mode=0)]:
+        with pytest.raises(lk.LckvError) as e:
+            cache.lckv_decode_attention(bad["slot"], bad["mode"], q)
+        assert e.value.status == lk.EINVAL
+    with pytest.raises(lk.LckvError) as e:
+        cache.lckv_cache_reset([9, 0])
+    assert e.value.status == lk.ECAPACITY
+    with pytest.raises(lk.LckvError) as e:
+        cache.lckv_layer_stack_step([q, q], [q, q], [None, None], [None, None])  # top k,v missing
+    assert e.value.status == lk.EINVAL
+    with pytest.raises(lk.LckvError) as e:
+        cache.lckv_decode_attention(0, 0, q, batch=3)
+    assert e.value.status == lk.EINVAL
+    cache.close()
+
+
+def test_host_buffer_entry_point_matches():
+    c = Case(L=4, w=2, Hq=8, Hkv=8, d=128, lens=[5, 100, 33], T_cap=120, seed=61, host_staging=1)
+    c.step(host=True); c.step(host=True)
+    c.close()
+
+
+def test_repeatable_bitwise():
+    """Same inputs twice: identical bits (the merge order is fixed, not arrival order)."""
+    outs = []
+    for _ in range(2):
+        c = Case(L=2, w=0, Hq=4, Hkv=4, d=128, lens=[3000, 700, 1234], T_cap=3001, seed=12)
+        o, _, _ = c.step()
+        outs.append([syn.bits(t) for t in o])
+        c.close()
+    for a, b in zip(*outs):
+        assert np.array_equal(a, b)
