@@ -1,0 +1,415 @@
+#!/usr/bin/env python
+"""Benchmark of the LCKV layer-stack decode step (one new token per sequence, all layers).
+
+A "step" is one lckv_layer_stack_step: plan, every layer's attention over its cache (the shared
+top-layer cache for condensed layers, own caches for warmup layers), the appends of the layers that
+have k,v, and the length advance.  The metric is the algorithmic KV bytes the step reads
+(sum over layers and sequences of 4*H_kv*d_h*visible rows) per second.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload llama7b] [--batch B]
+    python bench.py --impl reference ...     # times the float64 CPU checker on a bounded sample
+
+One JSON line is printed by rank 0.  With N > 1 (torchrun) every rank runs the same per-GPU
+workload on its own GPU (sequences are independent: no collective on the data path) and the
+value is the sum over ranks divided by the slowest rank's time.
+"""
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+import torch
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2405_10637_b200 import inputs as syn  # noqa: E402
+
+METRIC = "condensed decode-attn GB/s (% of 8 TB/s HBM) and layer-stack attn µs/step vs B"
+NOMINAL_HBM_GBS = 8000.0
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return 6650.0, "fallback"
+
+
+def workload_params(args):
+    wl = syn.WORKLOADS[args.workload]
+    if args.workload == "llama7b":
+        p = dict(batch=512, lo=256, hi=4096, t_cap=4096, sweep=[8, 16, 32, 64, 128, 256, 512])
+    elif args.workload == "tinyllama":
+        p = dict(batch=128, lo=1024, hi=1024, t_cap=1024, sweep=[128])
+    elif args.workload == "toy":
+        p = dict(batch=2, lo=128, hi=128, t_cap=128, sweep=[2])
+    elif args.workload == "llama30b":
+        p = dict(batch=256, lo=3072, hi=3072, t_cap=3072, sweep=[256])
+    elif args.workload == "sweep7b":
+        p = dict(batch=64, lo=8192, hi=8192, t_cap=8192, sweep=[64])
+    else:
+        raise SystemExit(f"unknown workload {args.workload}")
+    if args.batch:
+        p["batch"] = args.batch
+        p["sweep"] = [b for b in p["sweep"] if b <= args.batch] or [args.batch]
+        if args.batch not in p["sweep"]:
+            p["sweep"].append(args.batch)
+    if args.warmup_layers is not None:
+        wl = wl.with_(n_warmup=args.warmup_layers)
+    if args.context:
+        p["lo"] = p["hi"] = args.context
+        p["t_cap"] = args.context
+    # room for the tokens the run itself appends (lengths grow by one per step)
+    p["t_cap"] += max(64, args.steps + args.warmup + 8)
+    return wl, p
+
+
+def step_kv_bytes(wl, plan_modes, lens, batch, grown=0):
+    """Algorithmic K+V bytes one step reads: every layer reads its visible rows once.
+    `grown` = tokens appended to every sequence since `lens` was set."""
+    per_row = 4 * wl.n_kv_heads * wl.head_dim
+    s = int(np.asarray(lens[:batch], np.int64).sum()) + grown * batch
+    total = 0
+    for m in plan_modes:
+        total += per_row * (s + m * batch)
+    return total
+
+
+class ClockSampler:
+    """Samples nvidia-smi SM clocks and throttle reasons while the timed region runs."""
+
+    Q = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index):
+        self.index, self.rows, self.proc = index, [], None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(self.index), f"--query-gpu={self.Q}",
+                 "--format=csv,noheader,nounits", "-lms", "100"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append([x.strip() for x in line.split(",")])
+
+    def stop(self):
+        if not self.proc:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for r in self.rows:
+            try:
+                sm.append(float(r[0])); mx.append(float(r[1]))
+            except Exception:
+                continue
+            for n, v in zip(names, r[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        return {"sm_mhz": float(np.median(sm)) if sm else None,
+                "sm_max_mhz": max(mx) if mx else None, "reasons": sorted(reasons),
+                "samples": len(sm)}
+
+
+def oracle_sample(wl, plan, Ks, Vs, lens, rows, scale, min_seconds=10.0):
+    """Times the CPU checker, as it stands, on the first `rows` sequences (all layers)."""
+    from oracle import lckv_oracle as orc
+    L = wl.n_layers
+    q = [syn.bits(syn.randn_bf16((rows, wl.n_q_heads, wl.head_dim), 900 + l, std=wl.std))
+         for l in range(L)]
+    kv = [syn.bits(syn.randn_bf16((rows, wl.n_kv_heads, wl.head_dim), 950 + l, std=wl.std))
+          if plan["write_slot"][l] >= 0 else None for l in range(L)]
+    modes = [int(m) for m in plan["mode"]]
+    nbytes = step_kv_bytes(wl, modes, lens, rows)
+    t_total, n = 0.0, 0
+    while t_total < min_seconds and n < 50:
+        ln = np.asarray(lens[:rows], np.int32).copy()
+        t0 = time.perf_counter()
+        orc.stack_step(L, wl.n_warmup, q, kv, kv, Ks, Vs, ln, scale)
+        t_total += time.perf_counter() - t0
+        n += 1
+        # undo the append so that every repetition does the same work
+        # (the appended row lies beyond the restored length and is simply overwritten next time)
+    return nbytes * n / t_total / 1e9, orc.num_threads(), n, t_total / n
+
+
+def run_reference(args):
+    """--impl reference: the float64 CPU checker on a bounded sample of the same workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from oracle import lckv_oracle as orc
+    wl, p = workload_params(args)
+    rows = min(args.ref_rows, p["batch"])
+    lens = syn.ragged_lengths(p["batch"], p["lo"], p["hi"], syn.seed_for(wl, syn.T_LENS)).numpy()
+    plan = orc.plan(wl.n_layers, wl.n_warmup, 0)
+    scale = wl.head_dim ** -0.5
+    Ks = [syn.bits(syn.randn_bf16((rows, wl.n_kv_heads, p["t_cap"], wl.head_dim),
+                                   syn.seed_for(wl, syn.T_K, s), std=wl.std))
+          for s in range(plan["n_slots"])]
+    Vs = [syn.bits(syn.randn_bf16((rows, wl.n_kv_heads, p["t_cap"], wl.head_dim),
+                                   syn.seed_for(wl, syn.T_V, s), std=wl.std))
+          for s in range(plan["n_slots"])]
+    L = wl.n_layers
+    q = [syn.bits(syn.randn_bf16((rows, wl.n_q_heads, wl.head_dim), 900 + l, std=wl.std))
+         for l in range(L)]
+    kv = [syn.bits(syn.randn_bf16((rows, wl.n_kv_heads, wl.head_dim), 950 + l, std=wl.std))
+          if plan["write_slot"][l] >= 0 else None for l in range(L)]
+    modes = [int(m) for m in plan["mode"]]
+    nbytes = step_kv_bytes(wl, modes, lens, rows)
+
+    def one():
+        ln = np.asarray(lens[:rows], np.int32).copy()
+        t0 = time.perf_counter()
+        orc.stack_step(L, wl.n_warmup, q, kv, kv, Ks, Vs, ln, scale)
+        return time.perf_counter() - t0
+    for _ in range(args.warmup):
+        one()
+    ts = [one() for _ in range(args.steps)]
+    ms = 1e3 * float(np.mean(ts))
+    val = nbytes / (ms * 1e-3) / 1e9
+    sample = f"first {rows} of {p['batch']} sequences, all {L} layers, one decode step per step"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": val, "unit": "GB/s", "n_gpus": 0,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": workload_name(wl, p), "sample_rows": rows},
+        "cpu_baseline": {"value": val, "unit": "GB/s", "cores": orc.num_threads(),
+                         "kind": "oracle", "sample": sample},
+        "e2e": {"value": val, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def workload_name(wl, p):
+    ctx = f"ragged U[{p['lo']},{p['hi']}]" if p["lo"] != p["hi"] else f"context {p['lo']}"
+    return (f"{wl.name}: L={wl.n_layers} H_q={wl.n_q_heads} H_kv={wl.n_kv_heads} d_h={wl.head_dim} "
+            f"w={wl.n_warmup} {ctx} B={p['batch']} one decode step")
+
+
+def time_steps(fn, steps, stream):
+    """CUDA-event time of `steps` calls of fn on the current stream, in ms (total)."""
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream)
+    for _ in range(steps):
+        fn()
+    e1.record(stream)
+    e1.synchronize()
+    return e0.elapsed_time(e1)
+
+
+def run_ours(args):
+    from paper_2405_10637_b200 import binding as lk
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world != args.gpus and world > 1:
+        raise SystemExit("--gpus must equal WORLD_SIZE under torchrun")
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist = dist_
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    dev = torch.device(f"cuda:{local}")
+    stream = torch.cuda.current_stream()
+
+    wl, p = workload_params(args)
+    B, T_cap = p["batch"], p["t_cap"]
+    L = wl.n_layers
+    cfg = lk.make_config(L, wl.n_warmup, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, B, T_cap,
+                         host_staging=1, use_graph=1 if args.graph else 0,
+                         top_variant=args.top_variant)
+    cache = lk.Cache(cfg, device=dev)
+    plan = lk.lckv_plan(L, wl.n_warmup, args.top_variant)
+    info = cache.info
+    # every rank draws its own sequences (different seeds): independent replicas of the workload
+    lens = syn.ragged_lengths(B, p["lo"], p["hi"], syn.seed_for(wl, syn.T_LENS, rank)).numpy()
+    for s in range(info.n_slots):
+        kt, vt = cache.slot_tensors(s)
+        syn.fill_randn_bf16_(kt, syn.seed_for(wl, syn.T_K, s + 16 * rank), std=wl.std)
+        syn.fill_randn_bf16_(vt, syn.seed_for(wl, syn.T_V, s + 16 * rank), std=wl.std)
+    q = [syn.randn_bf16((B, wl.n_q_heads, wl.head_dim), 900 + l, device=dev, std=wl.std)
+         for l in range(L)]
+    kv = [syn.randn_bf16((B, wl.n_kv_heads, wl.head_dim), 950 + l, device=dev, std=wl.std)
+          if plan["write_slot"][l] >= 0 else None for l in range(L)]
+    outs = [torch.empty((B, wl.n_q_heads, wl.head_dim), dtype=torch.bfloat16, device=dev)
+            for _ in range(L)]
+    modes = plan["mode"]
+
+    def reset(b):
+        cache.lckv_cache_reset(lens[:b].tolist(), batch=b)
+
+    def make_step(b):
+        qs = [t[:b] for t in q]; os_ = [t[:b] for t in outs]
+        kvs = [None if t is None else t[:b] for t in kv]
+
+        def f():
+            cache.lckv_layer_stack_step(qs, os_, kvs, kvs, batch=b)
+        return f
+
+    def run_timed(f, b, warm, k):
+        """reset lengths, `warm` untimed steps, `k` timed steps (lengths grow by one per step).
+        Returns (ms per step, mean algorithmic bytes per timed step)."""
+        reset(b)
+        for _ in range(warm):
+            f()
+        barrier()
+        ms = time_steps(f, k, stream) / k
+        by = sum(step_kv_bytes(wl, modes, lens, b, warm + i) for i in range(k)) / k
+        return ms, by
+
+    def barrier():
+        torch.cuda.synchronize()
+        if dist:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def max_over_ranks(ms):
+        if not dist:
+            return ms
+        t = torch.tensor([ms], device=dev, dtype=torch.float64)
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        return float(t.item())
+
+    # ---- headline: K steps at the full batch --------------------------------------------------
+    step = make_step(B)
+    run_timed(step, B, 1, 1)  # first-touch of everything
+    sampler = ClockSampler(local)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+    ms_step, bytes_step = run_timed(step, B, args.warmup, args.steps)
+    barrier()
+    clocks = sampler.stop() if rank == 0 else None
+    ms_step = max_over_ranks(ms_step)
+    value = world * bytes_step / (ms_step * 1e-3) / 1e9
+    assert cache.lckv_cache_status() == 0, "device-side wait timed out"
+
+    # ---- roofline of the dominant kernel: condensed attention launches on the shared cache ------
+    n_launch = max(8, min(64, L))
+    qd, od = q[min(1, L - 1)], outs[min(1, L - 1)]
+
+    def attn():
+        cache.lckv_decode_attention(0, lk.MODE_CONDENSED, qd, out=od, batch=B)
+    reset(B)
+    for _ in range(3):
+        attn()
+    torch.cuda.synchronize()
+    ms_attn = time_steps(attn, n_launch, stream) / n_launch
+    io_bytes = 2 * B * wl.n_q_heads * wl.head_dim * 2
+    alg_bytes = 4 * wl.n_kv_heads * wl.head_dim * int(lens.astype(np.int64).sum()) + io_bytes
+    peak, peak_kind = measured_peaks()
+    achieved = alg_bytes / (ms_attn * 1e-3) / 1e9
+    roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                "frac": achieved / peak, "traffic": None, "peak_kind": peak_kind,
+                "kernel": "attn_alu_kernel" if info.kernel_kind == 1 else "attn_mma_kernel",
+                "us_per_launch": ms_attn * 1e3, "algorithmic_bytes_per_launch": alg_bytes,
+                "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
+
+    # ---- batch sweep (µs/step vs B) ---------------------------------------------------------
+    sweep = []
+    for b in p["sweep"]:
+        if b > B:
+            continue
+        f = make_step(b)
+        k = max(3, min(args.steps, 10))
+        ms, by = run_timed(f, b, 3, k)
+        ms = max_over_ranks(ms)
+        gbs = by / (ms * 1e-3) / 1e9
+        sweep.append({"B": b, "us_per_step": ms * 1e3, "kv_GBps": gbs,
+                      "frac_of_measured_peak": gbs / peak, "frac_of_8TBs": gbs / NOMINAL_HBM_GBS})
+
+    # ---- end to end through the host-buffer entry point ----------------------------------------
+    hq = [t.cpu().pin_memory() for t in q]
+    hkv = [None if t is None else t.cpu().pin_memory() for t in kv]
+    hout = [torch.empty((B, wl.n_q_heads, wl.head_dim), dtype=torch.bfloat16).pin_memory()
+            for _ in range(L)]
+
+    def e2e_step():
+        cache.lckv_layer_stack_step_host(hq, hout, hkv, hkv, batch=B)
+    k = max(3, min(args.steps, 10))
+    ms_e2e, by_e2e = run_timed(e2e_step, B, 3, k)
+    ms_e2e = max_over_ranks(ms_e2e)
+    h2d = sum(t.numel() * 2 for t in hq) + 2 * sum(t.numel() * 2 for t in hkv if t is not None)
+    d2h = sum(t.numel() * 2 for t in hout)
+    e2e = {"value": world * by_e2e / (ms_e2e * 1e-3) / 1e9, "unit": "GB/s",
+           "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e}
+
+    # ---- CPU baseline: the checker on a bounded sample (rank 0, N = 1 only) --------------------
+    cpu = None
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        rows = min(args.ref_rows, B)
+        Ks = [syn.bits(cache.slot_tensors(s)[0][:rows]) for s in range(info.n_slots)]
+        Vs = [syn.bits(cache.slot_tensors(s)[1][:rows]) for s in range(info.n_slots)]
+        gbs, cores, n, sec = oracle_sample(wl, {k_: np.asarray(v) for k_, v in plan.items()
+                                                if k_ != "n_slots"},
+                                           Ks, Vs, lens, rows, wl.head_dim ** -0.5)
+        cpu = {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
+               "sample": f"first {rows} of {B} sequences, all {L} layers, {n} repetitions of one "
+                         f"decode step ({sec:.2f} s each)"}
+
+    if rank == 0:
+        print(json.dumps({
+            "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+            "config": {"workload": workload_name(wl, p), "l2": "inputs larger than L2"
+                       if 2 * info.slot_bytes > 2 * 126e6 else "L2-resident cache: warm",
+                       "kv_bytes_per_step": bytes_step, "footprint_slots": info.n_slots,
+                       "top_variant": args.top_variant, "graph": bool(args.graph)},
+            "frac_of_8TBs": value / world / NOMINAL_HBM_GBS,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": info.launches_per_step * args.steps,
+            "roofline": roofline, "cpu_baseline": cpu, "sweep": sweep,
+        }))
+    cache.close()
+    if dist:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=10)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="llama7b", choices=sorted(syn.WORKLOADS))
+    ap.add_argument("--batch", type=int, default=0)
+    ap.add_argument("--context", type=int, default=0, help="equal context length for every sequence")
+    ap.add_argument("--warmup-layers", type=int, default=None, help="override w")
+    ap.add_argument("--top-variant", type=int, default=0)
+    ap.add_argument("--graph", type=int, default=1)
+    ap.add_argument("--ref-rows", type=int, default=32)
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        if not torch.cuda.is_available():
+            raise SystemExit("bench.py needs a CUDA device (the CUDA library has no CPU fallback)")
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

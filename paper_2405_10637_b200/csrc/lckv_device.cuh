@@ -51,7 +51,7 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait: false if the phase did not complete within `limit` polls (each poll may itself
 // block for a short hardware-defined time).
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
-                                                  uint32_t limit = (1u << 22))
+                                                  uint32_t limit = (1u << 20))
 {
     for (uint32_t it = 0; it < limit; ++it)
         if (mbar_try_wait(bar, parity)) return true;

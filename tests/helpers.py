@@ -18,7 +18,15 @@ def compare(got, want, what=""):
     assert np.isfinite(g).all(), f"{what}: non-finite GPU output"
     zero_rows = ~want.any(axis=-1)
     assert not g[zero_rows].any(), f"{what}: rows the oracle gives as exactly 0 are not 0"
-    max_abs = np.abs(g - want).max() if g.size else 0.0
+    err = np.abs(g - want)
+    max_abs = err.max() if g.size else 0.0
+    if got.dtype == torch.bfloat16:
+        # A bf16 output cannot be closer than half an ulp (2^-9 relative) to the true value, which
+        # exceeds 1e-2 once |o| > 5.12 and comes close to it from |o| = 4 on (short contexts with
+        # N(0,1) values do reach that).  Elements that large are allowed one bf16 ulp instead.
+        excess = err - np.maximum(MAX_ABS, np.abs(want) * 2.0 ** -8)
+        assert excess.max() <= 0, f"{what}: max-abs {max_abs:.3e} beyond tolerance and bf16 ulp"
+        max_abs = min(max_abs, MAX_ABS) if excess.max() <= 0 else max_abs
     denom = np.linalg.norm(want[~zero_rows])
     rel = np.linalg.norm((g - want)[~zero_rows]) / denom if denom > 0 else 0.0
     assert max_abs <= MAX_ABS, f"{what}: max-abs {max_abs:.3e}"
