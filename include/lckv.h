@@ -43,7 +43,8 @@ enum {
     LCKV_ECAPACITY = 2, /* a sequence would exceed max_seq rows                                */
     LCKV_ENOMEM = 3,    /* caller's buffer too small or not 256-byte aligned                   */
     LCKV_ECUDA = 4,     /* a CUDA runtime/driver call failed; see lckv_last_cuda_error         */
-    LCKV_ETIMEOUT = 5   /* a bounded device-side wait gave up (reported by lckv_cache_status)  */
+    LCKV_ETIMEOUT = 5,  /* a bounded device-side wait gave up (reported by lckv_cache_status)  */
+    LCKV_ESTATICLIMIT = 6 /* lckv_decode_attention_static: batch or GPU beyond its fixed scratch */
 };
 
 enum {
@@ -223,6 +224,55 @@ int lckv_layer_stack_step_host(lckv_cache_t* cache, const void* const* q_layers_
                                const void* const* k_new_layers_host,
                                const void* const* v_new_layers_host, int32_t batch,
                                void* stream);
+
+/*
+ * Decode attention without a cache object and without any allocation (the
+ * paper has no counterpart: this is a packaging variant of
+ * lckv_decode_attention for callers that cannot allocate).
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a
+ * serving engine that has already handed all device memory to its own pool,
+ * in a plugin whose host forbids allocation after initialisation, or on a
+ * latency path where an allocation's implicit synchronisation is not
+ * acceptable - and that also has nowhere to keep a workspace buffer for us.
+ * The regular entry point needs a caller-provided workspace for its work plan,
+ * split-K partials and merge tickets; this one keeps that scratch in a fixed
+ * array compiled into the library's device image instead.
+ *
+ * Same computation and argument meaning as lckv_decode_attention, with the
+ * cache described by plain pointers:
+ *   k, v      [batch, H_kv, max_seq, d_h] bf16, rows [0, visible) of each
+ *             (sequence, kv head) valid
+ *   lens      [batch] int32 DEVICE array, tokens cached per sequence
+ *   q, out, lse, mode, softmax_scale (0 => 1/sqrt(d_h)), out_dtype as above
+ *   dev_status  optional DEVICE int32: receives LCKV_ETIMEOUT if a bounded
+ *             device-side wait gave up (it is cleared to 0 first); NULL to ignore
+ * Limits: batch <= LCKV_STATIC_MAX_BATCH and a GPU with at most
+ * LCKV_STATIC_MAX_SMS multiprocessors, else LCKV_ESTATICLIMIT and nothing runs.
+ * The scratch array is LCKV_STATIC_SCRATCH_BYTES of device memory that every
+ * GPU loading this library holds until the process exits.
+ *
+ * Set-up: the first call on each device looks up the array's device address
+ * and raises the kernel's shared-memory limit; make that first call outside
+ * any stream capture.  Later calls on that device only enqueue work.
+ * Sharing: all calls on a device use the same scratch.  Calls are safe one
+ * after another on one stream (the merge tickets are cleared at the start of
+ * each call); calls that may overlap on the GPU - different streams, or a
+ * cache-based call is unaffected but two static calls are - race on it and
+ * give undefined results.  The lengths are read on the device, so a length
+ * beyond max_seq cannot be refused here: the caller guarantees
+ * 0 <= lens[b] and lens[b] + mode <= max_seq.
+ * This call performs no cudaMalloc/cudaFree and uses no allocating library.
+ * Errors: EINVAL (null pointer, bad shape or mode), ESTATICLIMIT, ECUDA.
+ */
+#define LCKV_STATIC_MAX_BATCH 4096
+#define LCKV_STATIC_MAX_SMS 256
+#define LCKV_STATIC_SCRATCH_BYTES (2304 * 1024)
+int lckv_decode_attention_static(const void* k, const void* v, const int32_t* lens,
+                                 const void* q, void* out, float* lse, int32_t* dev_status,
+                                 int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
+                                 int32_t head_dim, int64_t max_seq, int32_t mode,
+                                 float softmax_scale, int32_t out_dtype, void* stream);
 
 /* Short English name of a status code. */
 const char* lckv_status_string(int status);

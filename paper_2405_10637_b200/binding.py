@@ -11,7 +11,7 @@ import torch
 
 from . import build as _build
 
-OK, EINVAL, ECAPACITY, ENOMEM, ECUDA, ETIMEOUT = range(6)
+OK, EINVAL, ECAPACITY, ENOMEM, ECUDA, ETIMEOUT, ESTATICLIMIT = range(7)
 MODE_CONDENSED, MODE_STANDARD = 0, 1
 
 
@@ -47,6 +47,8 @@ SIGNATURES = {
     "lckv_decode_attention": (C.c_int, [_vp, _i32, _i32, _vp, _vp, _vp, _i32, _vp]),
     "lckv_layer_stack_step": (C.c_int, [_vp, _vpp, _vpp, _vpp, _vpp, _i32, _vp]),
     "lckv_layer_stack_step_host": (C.c_int, [_vp, _vpp, _vpp, _vpp, _vpp, _i32, _vp]),
+    "lckv_decode_attention_static": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32,
+                                              _i32, C.c_int64, _i32, C.c_float, _i32, _vp]),
     "lckv_status_string": (C.c_char_p, [C.c_int]),
     "lckv_last_cuda_error": (C.c_int, []),
 }
@@ -119,6 +121,22 @@ def make_config(n_layers, n_warmup, n_q_heads, n_kv_heads, head_dim, max_batch, 
 
 def lckv_cache_bytes(cfg):
     return int(lib().lckv_cache_bytes(C.byref(cfg)))
+
+
+def lckv_decode_attention_static(k, v, lens, q, out, mode, lse=None, dev_status=None,
+                                 softmax_scale=0.0, stream=None):
+    """Decode attention for callers that must not allocate: k, v [B, H_kv, T_cap, d_h] bf16,
+    lens [B] int32, q [B, H_q, d_h] bf16 and `out` (bf16 or fp32, caller-provided) are CUDA
+    tensors; the library's scratch is a fixed array inside its device image, so nothing is
+    allocated here or there.  One call at a time per GPU: all calls share that scratch."""
+    B, Hkv, T_cap, d = k.shape
+    Hq = q.shape[1]
+    rc = lib().lckv_decode_attention_static(
+        _ptr(k), _ptr(v), _ptr(lens), _ptr(q), _ptr(out), _ptr(lse), _ptr(dev_status), q.shape[0],
+        Hq, Hkv, d, T_cap, mode, softmax_scale, 1 if out.dtype == torch.float32 else 0,
+        _stream(stream))
+    _chk(rc, "lckv_decode_attention_static")
+    return out
 
 
 class Cache:

@@ -488,6 +488,7 @@ const char* lckv_status_string(int s)
         case LCKV_ENOMEM: return "device buffer too small or misaligned";
         case LCKV_ECUDA: return "CUDA call failed";
         case LCKV_ETIMEOUT: return "device-side wait timed out";
+        case LCKV_ESTATICLIMIT: return "size exceeds the static scratch of the no-allocation entry point";
         default: return "unknown status";
     }
 }
@@ -495,3 +496,117 @@ const char* lckv_status_string(int s)
 int lckv_last_cuda_error(void) { return g_last_cuda_error; }
 
 }  // extern "C"
+
+// =============================================================================================
+// Decode attention for callers that cannot allocate: scratch in a fixed device array.
+// =============================================================================================
+namespace {
+
+constexpr int kStaticMaxWorkers = LCKV_STATIC_MAX_SMS * lckv::kAluWarps;
+constexpr int kStaticPreStride = LCKV_STATIC_MAX_BATCH + 64;
+constexpr size_t kStOffPre = 0;
+constexpr size_t kStOffStart = kStOffPre + 2 * (size_t)kStaticPreStride * 4;
+constexpr size_t kStOffCounters = kStOffStart + 2 * (size_t)kStaticMaxWorkers * 4;
+constexpr size_t kStOffStatus = kStOffCounters + (size_t)kStaticMaxWorkers * 4;
+constexpr size_t kStOffPartials = kStOffStatus + 256;
+constexpr size_t kStBytes = kStOffPartials + 2 * (size_t)kStaticMaxWorkers * (128 + 4) * 4;
+static_assert(kStBytes <= LCKV_STATIC_SCRATCH_BYTES, "static scratch too small for its limits");
+static_assert(kStOffStart % 256 == 0 && kStOffCounters % 256 == 0 && kStOffPartials % 256 == 0,
+              "sections must stay 256-byte aligned");
+
+// Work plan, tickets, status word and split-K partials of lckv_decode_attention_static.  In host
+// code this name is only a handle for cudaGetSymbolAddress, never a pointer to pass to a kernel.
+static __device__ __align__(256) unsigned char g_static_scratch[LCKV_STATIC_SCRATCH_BYTES];
+
+constexpr int kMaxDevices = 64;
+unsigned char* g_static_ptr[kMaxDevices];   // device address of the array, per device
+int g_static_sms[kMaxDevices];
+
+// Once per device, with that device current: resolve the array's device address.
+int static_setup(int dev)
+{
+    void* ptr = nullptr;
+    if (!cuda_ok(cudaGetSymbolAddress(&ptr, g_static_scratch))) return LCKV_ECUDA;
+    if (!ptr) return LCKV_ECUDA;
+    int sms = 0;
+    if (!cuda_ok(cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev))) return LCKV_ECUDA;
+    if (!cuda_ok(cudaFuncSetAttribute(lckv::attn_alu_kernel<128>,
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      lckv::kAluSmemBytes)) ||
+        !cuda_ok(cudaFuncSetAttribute(lckv::attn_alu_kernel<64>,
+                                      cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      lckv::kAluSmemBytes)))
+        return LCKV_ECUDA;
+    g_static_sms[dev] = sms;
+    g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
+    return LCKV_OK;
+}
+
+}  // namespace
+
+extern "C" int lckv_decode_attention_static(const void* k, const void* v, const int32_t* lens,
+                                            const void* q, void* out, float* lse,
+                                            int32_t* dev_status, int32_t batch, int32_t n_q_heads,
+                                            int32_t n_kv_heads, int32_t head_dim, int64_t max_seq,
+                                            int32_t mode, float softmax_scale, int32_t out_dtype,
+                                            void* stream)
+{
+    if (!k || !v || !lens || !q || !out) return LCKV_EINVAL;
+    if (batch < 1 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads) return LCKV_EINVAL;
+    if (head_dim != 64 && head_dim != 128) return LCKV_EINVAL;
+    if (max_seq < 1 || (mode != LCKV_MODE_CONDENSED && mode != LCKV_MODE_STANDARD)) return LCKV_EINVAL;
+    if (out_dtype != 0 && out_dtype != 1) return LCKV_EINVAL;
+    if (!(softmax_scale >= 0.f) || !std::isfinite(softmax_scale)) return LCKV_EINVAL;
+    if (batch > LCKV_STATIC_MAX_BATCH) return LCKV_ESTATICLIMIT;
+    if ((uint64_t)batch * (((uint64_t)max_seq + 15) / 16) >= (1ull << 31)) return LCKV_EINVAL;
+    int dev = 0;
+    if (!cuda_ok(cudaGetDevice(&dev))) return LCKV_ECUDA;
+    if (dev < 0 || dev >= kMaxDevices) return LCKV_ESTATICLIMIT;
+    if (!g_static_ptr[dev])
+        if (int rc = static_setup(dev)) return rc;
+    const int sms = g_static_sms[dev];
+    if (sms > LCKV_STATIC_MAX_SMS) return LCKV_ESTATICLIMIT;
+    unsigned char* base = g_static_ptr[dev];
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    const int n_workers = sms * lckv::kAluWarps;
+    uint32_t* d_pre = reinterpret_cast<uint32_t*>(base + kStOffPre);
+    int32_t* d_start = reinterpret_cast<int32_t*>(base + kStOffStart);
+    int32_t* d_counters = reinterpret_cast<int32_t*>(base + kStOffCounters);
+    int32_t* d_status = dev_status ? dev_status : reinterpret_cast<int32_t*>(base + kStOffStatus);
+
+    // The array keeps whatever the previous call left: the tickets must start at zero.
+    if (!cuda_ok(cudaMemsetAsync(d_counters, 0, (size_t)n_workers * 4, st))) return LCKV_ECUDA;
+    if (!cuda_ok(cudaMemsetAsync(d_status, 0, 4, st))) return LCKV_ECUDA;
+
+    const int R = lckv::kAluSlotBytes / (head_dim * 2);
+    lckv::plan_kernel<<<1, 1024, 0, st>>>(lens, batch, R, n_q_heads, n_workers, d_pre,
+                                          kStaticPreStride, d_start);
+    if (!cuda_ok(cudaGetLastError())) return LCKV_ECUDA;
+
+    lckv::AttnParams p;
+    p.K = static_cast<const uint16_t*>(k);
+    p.V = static_cast<const uint16_t*>(v);
+    p.q = static_cast<const uint16_t*>(q);
+    p.out = out;
+    p.lse = lse;
+    p.lens = lens;
+    p.pre = d_pre + (size_t)mode * kStaticPreStride;
+    p.start_b = d_start + (size_t)mode * n_workers;
+    p.partials = reinterpret_cast<float*>(base + kStOffPartials);
+    p.counters = d_counters;
+    p.status = d_status;
+    p.T_cap = max_seq;
+    p.B = batch;
+    p.H_q = n_q_heads;
+    p.H_kv = n_kv_heads;
+    p.mode = mode;
+    p.n_workers = n_workers;
+    p.out_f32 = out_dtype;
+    const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
+    p.scale_log2 = scale * 1.4426950408889634f;
+    if (head_dim == 128)
+        lckv::attn_alu_kernel<128><<<sms, lckv::kAluWarps * 32, lckv::kAluSmemBytes, st>>>(p);
+    else
+        lckv::attn_alu_kernel<64><<<sms, lckv::kAluWarps * 32, lckv::kAluSmemBytes, st>>>(p);
+    return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
+}
