@@ -9,6 +9,7 @@
 
 #include "../../include/lckv.h"
 #include "lckv_attn_alu.cuh"
+#include "lckv_attn_mma.cuh"
 #include "lckv_small_kernels.cuh"
 
 namespace {
@@ -86,6 +87,7 @@ struct lckv_cache {
     float* d_partials;
     std::vector<int32_t> h_lens;  // host mirror of the device lengths
     int n_kv_layers;
+    std::vector<CUtensorMap> tm_k, tm_v;  // per slot, tensor-core kernel only
 };
 
 namespace {
@@ -108,7 +110,49 @@ int validate_config(const lckv_config_t* c)
     return LCKV_OK;
 }
 
-int resolve_kernel_kind(const lckv_config_t&) { return 1; }
+// 1 = FP32-ALU kernel, 2 = tensor-core kernel (query groups that are multiples of 8).
+int resolve_kernel_kind(const lckv_config_t& c)
+{
+    const int g = c.n_q_heads / c.n_kv_heads;
+    return (c.kernel_kind == 0 && g % 8 == 0) ? 2 : 1;
+}
+
+int partial_record_floats(const lckv_config_t& c)
+{
+    return resolve_kernel_kind(c) == 2 ? c.head_dim * 8 + 16 : c.head_dim + 4;
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*,
+                                  const cuuint64_t*, const cuuint64_t*, const cuuint32_t*,
+                                  const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+// Tensor map of one K or V tensor seen as [rows = B_max*H_kv*T_cap, d_h] bf16, box = 64 columns x
+// `box_rows` rows, 128-byte swizzle, out-of-range rows read as zero.
+int make_tensor_map(CUtensorMap* tm, void* base, uint64_t rows, int d, int box_rows)
+{
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void* f = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (!cuda_ok(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f, cudaEnableDefault, &q)))
+            return LCKV_ECUDA;
+        if (q != cudaDriverEntryPointSuccess || !f) return LCKV_ECUDA;
+        fn = reinterpret_cast<EncodeTiledFn>(f);
+    }
+    const cuuint64_t gdim[2] = {(cuuint64_t)d, (cuuint64_t)rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)d * 2};
+    const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box, estr,
+                          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                          CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        g_last_cuda_error = (int)r;
+        return LCKV_ECUDA;
+    }
+    return LCKV_OK;
+}
 
 void make_layout(const lckv_config_t& c, int n_slots, int n_workers, int n_kv_layers, Layout& y)
 {
@@ -120,7 +164,8 @@ void make_layout(const lckv_config_t& c, int n_slots, int n_workers, int n_kv_la
     y.off_start = off;     off = align_up(off + 2 * (size_t)n_workers * 4, A);
     y.off_counters = off;  off = align_up(off + (size_t)n_workers * 4, A);
     y.off_status = off;    off = align_up(off + 4, A);
-    y.off_partials = off;  off = align_up(off + 2 * (size_t)n_workers * (c.head_dim + 4) * 4, A);
+    y.off_partials = off;
+    off = align_up(off + 2 * (size_t)n_workers * partial_record_floats(c) * 4, A);
     y.workspace_bytes = off;
     y.slot_bytes =
         align_up((size_t)c.max_batch * c.n_kv_heads * (size_t)c.max_seq * c.head_dim * 2, A);
@@ -193,10 +238,23 @@ int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out
     p.n_workers = c->n_workers;
     p.out_f32 = c->cfg.out_dtype;
     p.scale_log2 = c->scale_log2;
-    if (c->cfg.head_dim == 128)
+    if (c->kernel_kind == 2) {
+        lckv::MmaParams mp;
+        mp.a = p;
+        mp.a.H_q = c->h_pairs;  // pairs per sequence = groups of 8 query heads
+        mp.n_q_heads = c->cfg.n_q_heads;
+        mp.groups_per_kv = c->cfg.n_q_heads / c->cfg.n_kv_heads / 8;
+        if (c->cfg.head_dim == 128)
+            lckv::attn_mma_kernel<128><<<c->grid, lckv::kMmaWarps * 32, lckv::kMmaSmemBytes, st>>>(
+                mp, c->tm_k[slot], c->tm_v[slot]);
+        else
+            lckv::attn_mma_kernel<64><<<c->grid, lckv::kMmaWarps * 32, lckv::kMmaSmemBytes, st>>>(
+                mp, c->tm_k[slot], c->tm_v[slot]);
+    } else if (c->cfg.head_dim == 128) {
         lckv::attn_alu_kernel<128><<<c->grid, lckv::kAluWarps * 32, lckv::kAluSmemBytes, st>>>(p);
-    else
+    } else {
         lckv::attn_alu_kernel<64><<<c->grid, lckv::kAluWarps * 32, lckv::kAluSmemBytes, st>>>(p);
+    }
     return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
 }
 
@@ -295,7 +353,7 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     c->n_workers = sm * lckv::kAluWarps;
     c->kernel_kind = resolve_kernel_kind(*cfg);
     c->rows_per_tile = lckv::kAluSlotBytes / (cfg->head_dim * 2);
-    c->h_pairs = cfg->n_q_heads;
+    c->h_pairs = c->kernel_kind == 2 ? cfg->n_q_heads / 8 : cfg->n_q_heads;
     make_layout(*cfg, c->plan.n_slots, c->n_workers, c->n_kv_layers, c->lay);
     if (dev_bytes < c->lay.total_bytes) { delete c; return LCKV_ENOMEM; }
     const float scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale
@@ -310,7 +368,23 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     c->d_partials = reinterpret_cast<float*>(c->base + c->lay.off_partials);
     c->h_lens.assign(cfg->max_batch, 0);
 
-    bool ok = cuda_ok(cudaFuncSetAttribute(lckv::attn_alu_kernel<128>,
+    if (c->kernel_kind == 2) {
+        const uint64_t rows = (uint64_t)cfg->max_batch * cfg->n_kv_heads * (uint64_t)cfg->max_seq;
+        c->tm_k.resize(c->plan.n_slots);
+        c->tm_v.resize(c->plan.n_slots);
+        for (int s = 0; s < c->plan.n_slots; ++s) {
+            int rc = make_tensor_map(&c->tm_k[s], slot_k(c, s), rows, cfg->head_dim, c->rows_per_tile);
+            if (!rc) rc = make_tensor_map(&c->tm_v[s], slot_v(c, s), rows, cfg->head_dim, c->rows_per_tile);
+            if (rc) { delete c; return rc; }
+        }
+    }
+    bool ok = cuda_ok(cudaFuncSetAttribute(lckv::attn_mma_kernel<128>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           lckv::kMmaSmemBytes)) &&
+              cuda_ok(cudaFuncSetAttribute(lckv::attn_mma_kernel<64>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           lckv::kMmaSmemBytes)) &&
+              cuda_ok(cudaFuncSetAttribute(lckv::attn_alu_kernel<128>,
                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            lckv::kAluSmemBytes)) &&
               cuda_ok(cudaFuncSetAttribute(lckv::attn_alu_kernel<64>,

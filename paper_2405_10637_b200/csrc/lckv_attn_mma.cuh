@@ -1,0 +1,416 @@
+// Decode attention, tensor-core kernel for grouped-query attention: the 8 query heads that share a
+// kv head form the N = 8 side of a dense bf16 m16n8k16 MMA tile.
+//
+//   S^T [tokens x 8] = K [tokens x d] . Q^T [d x 8]        (tokens are the M dimension)
+//   O^T [d x 8]      = V^T [d x tokens] . P^T [tokens x 8]
+//
+// Work decomposition, per-warp copy ring, running-max softmax and the ticketed merge of split
+// pairs are those of the FP32-ALU kernel (lckv_attn_alu.cuh); a pair here is (sequence, group of 8
+// query heads).  Differences: tiles arrive through 2-D tiled TMA with the 128-byte swizzle so that
+// ldmatrix reads them without bank conflicts; the probabilities are rounded to bf16 for the second
+// MMA (their sum is taken over the rounded values, so the weights stay normalised); a TMA box is
+// always whole, so rows past the visible count are fetched, masked in the scores and zeroed in V.
+#pragma once
+#include <cuda.h>
+
+#include "lckv_attn_alu.cuh"
+
+namespace lckv {
+
+constexpr int kMmaWarps = 8;
+constexpr int kMmaSlots = 6;
+constexpr int kMmaSlotBytes = 4096;
+constexpr int kMmaSmemBytes = kMmaWarps * kMmaSlots * (kMmaSlotBytes + 8) + 1024;  // + alignment slack
+
+__device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
+                                            uint32_t& r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr)
+                 : "memory");
+}
+
+__device__ __forceinline__ void ldmatrix_x4_trans(uint32_t addr, uint32_t& r0, uint32_t& r1,
+                                                  uint32_t& r2, uint32_t& r3)
+{
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.trans.shared.b16 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(r0), "=r"(r1), "=r"(r2), "=r"(r3)
+                 : "r"(addr)
+                 : "memory");
+}
+
+__device__ __forceinline__ uint32_t movmatrix_trans(uint32_t a)
+{
+    uint32_t d;
+    asm volatile("movmatrix.sync.aligned.m8n8.trans.b16 %0, %1;" : "=r"(d) : "r"(a));
+    return d;
+}
+
+__device__ __forceinline__ void mma_bf16_16816(float (&c)[4], uint32_t a0, uint32_t a1, uint32_t a2,
+                                               uint32_t a3, uint32_t b0, uint32_t b1)
+{
+    asm volatile(
+        "mma.sync.aligned.m16n8k16.row.col.f32.bf16.bf16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, "
+        "{%8,%9}, {%0,%1,%2,%3};"
+        : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+        : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// {lo, hi} -> packed bf16x2 (round to nearest even), lo in the low half.
+__device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi)
+{
+    uint32_t d;
+    asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
+    return d;
+}
+
+struct MmaParams {
+    AttnParams a;     // H_q here = pairs per sequence (groups of 8 query heads); see the launcher
+    int32_t n_q_heads;  // real H_q, for addressing q / out / lse
+    int32_t groups_per_kv;  // groups of 8 query heads that share one kv head
+};
+
+template <int D>
+__global__ void __launch_bounds__(kMmaWarps * 32, 1)
+attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
+                const __grid_constant__ CUtensorMap tmV)
+{
+    constexpr int R = kMmaSlotBytes / (D * 2);  // tokens per tile: 32 (D=64), 16 (D=128)
+    constexpr int RB = R / 16;                  // 16-token row blocks per tile
+    constexpr int KS = D / 16;                  // k-steps of the score MMA
+    constexpr int MT = D / 16;                  // 16-dim m-tiles of the output MMA
+    constexpr int NBOX = D / 64;                // 128-byte-wide TMA boxes per tile
+    constexpr int BOX_BYTES = R * 128;
+    constexpr int NS = kMmaSlots;
+    constexpr int REC = D * 8 + 16;             // floats per partial record
+    const AttnParams& p = mp.a;
+
+    extern __shared__ uint8_t smem_raw[];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int w = blockIdx.x * kMmaWarps + warp;
+    const int H = p.H_q;  // pairs per sequence
+    const uint32_t FULL = 0xffffffffu;
+    const int g4 = lane >> 2, c4 = lane & 3;
+
+    const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms are 1024 bytes
+    const uint32_t ring = smem0 + warp * (NS * kMmaSlotBytes);
+    const uint32_t bars = smem0 + kMmaWarps * NS * kMmaSlotBytes + warp * (NS * 8);
+    if (lane == 0) {
+        for (int s = 0; s < NS; ++s) mbar_init(bars + 8 * s, 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+
+    // Sequences that see nothing: zero rows (zero dummy KV), lse 0.
+    for (int b = w; b < p.B; b += p.n_workers) {
+        if (__ldg(p.lens + b) + p.mode == 0) {
+            const int esz = p.out_f32 ? 4 : 2;
+            const int n16 = mp.n_q_heads * D * esz / 16;
+            uint4* o16 = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.out) +
+                                                  (size_t)b * mp.n_q_heads * D * esz);
+            for (int i = lane; i < n16; i += 32) o16[i] = make_uint4(0, 0, 0, 0);
+            if (p.lse)
+                for (int i = lane; i < mp.n_q_heads; i += 32)
+                    p.lse[(size_t)b * mp.n_q_heads + i] = 0.f;
+        }
+    }
+
+    const uint64_t total = (uint64_t)__ldg(p.pre + p.B) * (uint64_t)H;
+    if (total == 0) return;
+    const uint64_t n_eff = total < (uint64_t)p.n_workers ? total : (uint64_t)p.n_workers;
+    if ((uint64_t)w >= n_eff) return;
+    const uint64_t lo = (uint64_t)w * total / n_eff;
+    const uint64_t hi = (uint64_t)(w + 1) * total / n_eff;
+    const uint32_t n_tiles = (uint32_t)(hi - lo);
+    const uint32_t n_items = 2 * n_tiles;
+
+    TileCursor cc;
+    cc.b = __ldg(p.start_b + w);
+    cursor_load(cc, p);
+    {
+        const uint64_t rel = lo - (uint64_t)__ldg(p.pre + cc.b) * (uint64_t)H;
+        cc.h = (int32_t)(rel / cc.nt);
+        cc.t = (uint32_t)(rel % cc.nt);
+    }
+    TileCursor ci = cc;
+
+    uint32_t issued = 0, islot = 0;
+    auto issue = [&]() {
+        const int kvh = ci.h / mp.groups_per_kv;
+        const int64_t row = ((int64_t)ci.b * p.H_kv + kvh) * p.T_cap + (int64_t)ci.t * R;
+        if (lane == 0) {
+            const void* tm = (issued & 1) ? (const void*)&tmV : (const void*)&tmK;
+            mbar_expect_tx(bars + 8 * islot, kMmaSlotBytes);
+#pragma unroll
+            for (int bx = 0; bx < NBOX; ++bx)
+                tma_load_2d(ring + islot * kMmaSlotBytes + bx * BOX_BYTES, tm, bx * 64, (int32_t)row,
+                            bars + 8 * islot);
+        }
+        if (issued & 1) cursor_next(ci, p, H);
+        ++issued;
+        islot = (islot + 1 == NS) ? 0 : islot + 1;
+    };
+    {
+        const uint32_t pro = n_items < (uint32_t)NS ? n_items : (uint32_t)NS;
+        while (issued < pro) issue();
+    }
+
+    uint32_t cslot = 0, cphase = 0;
+    bool ok = true;
+
+    // Q^T fragments of the pair's 8 query heads: lane holds query g4, dims 2*c4 (+1) (+8) per k-step.
+    uint32_t qb[KS][2];
+    auto load_q = [&](const TileCursor& c) {
+        const uint16_t* qp = p.q + ((size_t)c.b * mp.n_q_heads + (size_t)c.h * 8 + g4) * D + 2 * c4;
+#pragma unroll
+        for (int ks = 0; ks < KS; ++ks) {
+            qb[ks][0] = __ldg(reinterpret_cast<const uint32_t*>(qp + ks * 16));
+            qb[ks][1] = __ldg(reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8));
+        }
+    };
+    load_q(cc);
+    uint32_t seg_t0 = cc.t;
+    // running state for this lane's two queries (2*c4, 2*c4+1)
+    float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
+    float o[MT][4];
+#pragma unroll
+    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+        for (int i = 0; i < 4; ++i) o[mt][i] = 0.f;
+
+    for (uint32_t tile = 0; tile < n_tiles; ++tile) {
+        const int rows = min(R, cc.nv - (int)cc.t * R);
+
+        // ---- K tile: S^T = K . Q^T ----------------------------------------------------------
+        if (!mbar_wait_bounded(bars + 8 * cslot, cphase)) { ok = false; break; }
+        float s[RB][4];
+        {
+            const uint32_t slot = ring + cslot * kMmaSlotBytes;
+#pragma unroll
+            for (int rb = 0; rb < RB; ++rb) {
+#pragma unroll
+                for (int i = 0; i < 4; ++i) s[rb][i] = 0.f;
+                const int r = rb * 16 + (lane & 15);
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) {
+                    const int cg = 2 * ks + (lane >> 4);  // 16-byte chunk of the d-row
+                    const uint32_t addr = slot + (cg >> 3) * BOX_BYTES + r * 128 +
+                                          (((cg & 7) ^ (r & 7)) << 4);
+                    uint32_t a0, a1, a2, a3;
+                    ldmatrix_x4(addr, a0, a1, a2, a3);
+                    mma_bf16_16816(s[rb], a0, a1, a2, a3, qb[ks][0], qb[ks][1]);
+                }
+            }
+        }
+        __syncwarp();
+        if (issued < n_items) issue();
+        cslot = (cslot + 1 == NS) ? 0 : cslot + 1;
+        if (cslot == 0) cphase ^= 1;
+
+        // scale to base-2 logits, mask rows past the visible count
+        float mt_[2] = {-INFINITY, -INFINITY};
+#pragma unroll
+        for (int rb = 0; rb < RB; ++rb) {
+            const int t0 = rb * 16 + g4, t1 = t0 + 8;
+            s[rb][0] = (t0 < rows) ? s[rb][0] * p.scale_log2 : -INFINITY;
+            s[rb][1] = (t0 < rows) ? s[rb][1] * p.scale_log2 : -INFINITY;
+            s[rb][2] = (t1 < rows) ? s[rb][2] * p.scale_log2 : -INFINITY;
+            s[rb][3] = (t1 < rows) ? s[rb][3] * p.scale_log2 : -INFINITY;
+            mt_[0] = fmaxf(mt_[0], fmaxf(s[rb][0], s[rb][2]));
+            mt_[1] = fmaxf(mt_[1], fmaxf(s[rb][1], s[rb][3]));
+        }
+#pragma unroll
+        for (int off = 4; off <= 16; off <<= 1) {
+            mt_[0] = fmaxf(mt_[0], __shfl_xor_sync(FULL, mt_[0], off));
+            mt_[1] = fmaxf(mt_[1], __shfl_xor_sync(FULL, mt_[1], off));
+        }
+        float alpha[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const float m_new = fmaxf(m_run[j], mt_[j]);
+            alpha[j] = ex2(m_run[j] - m_new);
+            m_run[j] = m_new;
+            l_run[j] *= alpha[j];
+        }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt) {
+            o[mt][0] *= alpha[0]; o[mt][1] *= alpha[1];
+            o[mt][2] *= alpha[0]; o[mt][3] *= alpha[1];
+        }
+        // probabilities -> bf16 pairs -> transposed into the B operand of the second MMA
+        uint32_t pb[RB][2];
+#pragma unroll
+        for (int rb = 0; rb < RB; ++rb) {
+            const uint32_t lo_pack = cvt_bf16x2(ex2(s[rb][0] - m_run[0]), ex2(s[rb][1] - m_run[1]));
+            const uint32_t hi_pack = cvt_bf16x2(ex2(s[rb][2] - m_run[0]), ex2(s[rb][3] - m_run[1]));
+            l_run[0] += bf16lo(lo_pack) + bf16lo(hi_pack);
+            l_run[1] += bf16hi(lo_pack) + bf16hi(hi_pack);
+            pb[rb][0] = movmatrix_trans(lo_pack);
+            pb[rb][1] = movmatrix_trans(hi_pack);
+        }
+
+        // ---- V tile: O^T += V^T . P^T -------------------------------------------------------
+        if (!mbar_wait_bounded(bars + 8 * cslot, cphase)) { ok = false; break; }
+        {
+            const uint32_t slot = ring + cslot * kMmaSlotBytes;
+            if (rows < R) {
+                // rows past the visible count came along with the box: weight 0, but 0 * NaN = NaN
+#pragma unroll
+                for (int bx = 0; bx < NBOX; ++bx)
+                    for (int i = rows * 128 + lane * 16; i < BOX_BYTES; i += 32 * 16)
+                        sts128(slot + bx * BOX_BYTES + i, make_uint4(0, 0, 0, 0));
+                fence_proxy_async_smem();
+                __syncwarp();
+            }
+#pragma unroll
+            for (int rb = 0; rb < RB; ++rb) {
+                const int r = rb * 16 + (lane & 7) + ((lane >> 4) & 1) * 8;
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt) {
+                    const int cg = 2 * mt + ((lane >> 3) & 1);
+                    const uint32_t addr = slot + (cg >> 3) * BOX_BYTES + r * 128 +
+                                          (((cg & 7) ^ (r & 7)) << 4);
+                    uint32_t a0, a1, a2, a3;
+                    ldmatrix_x4_trans(addr, a0, a1, a2, a3);
+                    mma_bf16_16816(o[mt], a0, a1, a2, a3, pb[rb][0], pb[rb][1]);
+                }
+            }
+        }
+        __syncwarp();
+        if (issued < n_items) issue();
+        cslot = (cslot + 1 == NS) ? 0 : cslot + 1;
+        if (cslot == 0) cphase ^= 1;
+
+        // ---- end of this worker's part of the pair? -----------------------------------------
+        const bool pair_end = (cc.t + 1 == cc.nt);
+        const bool last = (tile + 1 == n_tiles);
+        if (pair_end || last) {
+            float l_tot[2] = {l_run[0], l_run[1]};
+#pragma unroll
+            for (int off = 4; off <= 16; off <<= 1) {
+                l_tot[0] += __shfl_xor_sync(FULL, l_tot[0], off);
+                l_tot[1] += __shfl_xor_sync(FULL, l_tot[1], off);
+            }
+            float m_fin[2] = {m_run[0], m_run[1]};
+
+            const bool complete = pair_end && seg_t0 == 0;
+            bool write_row = complete;
+            if (!complete) {
+                const uint64_t gs = (uint64_t)__ldg(p.pre + cc.b) * (uint64_t)H +
+                                    (uint64_t)cc.h * cc.nt;
+                const uint64_t ge = gs + cc.nt;
+                const uint32_t c_first = (uint32_t)(((gs + 1) * n_eff - 1) / total);
+                const uint32_t c_last = (uint32_t)((ge * n_eff - 1) / total);
+                const bool at_lo = (gs + seg_t0 == lo);
+                float* rec = p.partials + (size_t)(2 * w + (at_lo ? 0 : 1)) * REC;
+                // accumulators in fragment order: fully coalesced
+#pragma unroll
+                for (int mt = 0; mt < MT; ++mt)
+                    reinterpret_cast<float4*>(rec)[mt * 32 + lane] =
+                        make_float4(o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
+                if (g4 == 0) {
+                    rec[D * 8 + 2 * c4] = m_fin[0];     rec[D * 8 + 2 * c4 + 1] = m_fin[1];
+                    rec[D * 8 + 8 + 2 * c4] = l_tot[0]; rec[D * 8 + 8 + 2 * c4 + 1] = l_tot[1];
+                }
+                __threadfence();
+                __syncwarp();
+                int ticket = 0;
+                if (lane == 0) ticket = atomicAdd(p.counters + c_first, 1);
+                ticket = __shfl_sync(FULL, ticket, 0);
+                if (ticket == (int)(c_last - c_first)) {
+                    __threadfence();
+                    float M[2] = {-INFINITY, -INFINITY};
+                    for (uint32_t c = c_first; c <= c_last; ++c) {
+                        const uint64_t lo_c = (uint64_t)c * total / n_eff;
+                        const float* r = p.partials +
+                            (size_t)(2 * c + ((c == c_first && gs != lo_c) ? 1 : 0)) * REC;
+                        M[0] = fmaxf(M[0], __ldcg(r + D * 8 + 2 * c4));
+                        M[1] = fmaxf(M[1], __ldcg(r + D * 8 + 2 * c4 + 1));
+                    }
+                    float Ls[2] = {0.f, 0.f};
+                    float acc[MT][4];
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
+                    for (uint32_t c = c_first; c <= c_last; ++c) {
+                        const uint64_t lo_c = (uint64_t)c * total / n_eff;
+                        const float* r = p.partials +
+                            (size_t)(2 * c + ((c == c_first && gs != lo_c) ? 1 : 0)) * REC;
+                        const float w0 = ex2(__ldcg(r + D * 8 + 2 * c4) - M[0]);
+                        const float w1 = ex2(__ldcg(r + D * 8 + 2 * c4 + 1) - M[1]);
+                        Ls[0] = fmaf(__ldcg(r + D * 8 + 8 + 2 * c4), w0, Ls[0]);
+                        Ls[1] = fmaf(__ldcg(r + D * 8 + 8 + 2 * c4 + 1), w1, Ls[1]);
+#pragma unroll
+                        for (int mt = 0; mt < MT; ++mt) {
+                            const float4 x = __ldcg(reinterpret_cast<const float4*>(r) + mt * 32 + lane);
+                            acc[mt][0] = fmaf(x.x, w0, acc[mt][0]);
+                            acc[mt][1] = fmaf(x.y, w1, acc[mt][1]);
+                            acc[mt][2] = fmaf(x.z, w0, acc[mt][2]);
+                            acc[mt][3] = fmaf(x.w, w1, acc[mt][3]);
+                        }
+                    }
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                        for (int i = 0; i < 4; ++i) o[mt][i] = acc[mt][i];
+                    l_tot[0] = Ls[0]; l_tot[1] = Ls[1];
+                    m_fin[0] = M[0]; m_fin[1] = M[1];
+                    write_row = true;
+                    if (lane == 0) p.counters[c_first] = 0;
+                }
+            }
+            if (write_row) {
+                const float inv0 = 1.0f / l_tot[0], inv1 = 1.0f / l_tot[1];
+                const size_t row0 = (size_t)cc.b * mp.n_q_heads + (size_t)cc.h * 8;  // first q head
+                if (p.out_f32) {
+                    float* ob = static_cast<float*>(p.out);
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt) {
+                        const int d0 = mt * 16 + g4;
+                        ob[(row0 + 2 * c4) * D + d0] = o[mt][0] * inv0;
+                        ob[(row0 + 2 * c4 + 1) * D + d0] = o[mt][1] * inv1;
+                        ob[(row0 + 2 * c4) * D + d0 + 8] = o[mt][2] * inv0;
+                        ob[(row0 + 2 * c4 + 1) * D + d0 + 8] = o[mt][3] * inv1;
+                    }
+                } else {
+                    // transpose the [dims x queries] fragments so a lane holds two adjacent dims of
+                    // one query: 4-byte stores, one query row per 8 lanes
+                    uint16_t* ob = static_cast<uint16_t*>(p.out) + (row0 + g4) * D + 2 * c4;
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt) {
+                        const uint32_t t0 = movmatrix_trans(cvt_bf16x2(o[mt][0] * inv0, o[mt][1] * inv1));
+                        const uint32_t t1 = movmatrix_trans(cvt_bf16x2(o[mt][2] * inv0, o[mt][3] * inv1));
+                        *reinterpret_cast<uint32_t*>(ob + mt * 16) = t0;
+                        *reinterpret_cast<uint32_t*>(ob + mt * 16 + 8) = t1;
+                    }
+                }
+                if (p.lse && g4 == 0) {
+                    p.lse[row0 + 2 * c4] = (m_fin[0] + lg2(l_tot[0])) * 0.6931471805599453f;
+                    p.lse[row0 + 2 * c4 + 1] = (m_fin[1] + lg2(l_tot[1])) * 0.6931471805599453f;
+                }
+            }
+            m_run[0] = m_run[1] = -INFINITY;
+            l_run[0] = l_run[1] = 0.f;
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+                for (int i = 0; i < 4; ++i) o[mt][i] = 0.f;
+        }
+        if (!last) {
+            cursor_next(cc, p, H);
+            if (pair_end) { load_q(cc); seg_t0 = 0; }
+        }
+    }
+
+    if (!ok) {
+        if (lane == 0) atomicExch(p.status, kStatusTimeout);
+        for (int s = 0; s < NS; ++s) {
+            mbar_wait_bounded(bars + 8 * s, 0, 1u << 10);
+            mbar_wait_bounded(bars + 8 * s, 1, 1u << 10);
+        }
+    }
+}
+
+}  // namespace lckv

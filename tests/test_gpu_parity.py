@@ -174,3 +174,47 @@ def test_repeatable_bitwise():
         c.close()
     for a, b in zip(*outs):
         assert np.array_equal(a, b)
+
+
+# ---- tensor-core kernel (query groups that are multiples of 8) -----------------------------------
+
+@pytest.mark.parametrize("d,Hq,Hkv", [(64, 32, 4), (128, 16, 2), (64, 32, 2), (128, 8, 1)])
+def test_mma_kernel_edge_lengths(d, Hq, Hkv):
+    lens = [0, 1, 15, 16, 17, 31, 32, 33, 47, 48, 49, 64, 100, 257, 300]
+    c = Case(L=4, w=2, Hq=Hq, Hkv=Hkv, d=d, lens=lens, T_cap=303, seed=500 + d + Hq, std=0.5)
+    assert c.cache.info.kernel_kind == 2
+    for _ in range(3):
+        c.step()
+    c.close()
+
+
+def test_mma_kernel_many_pairs_per_worker_and_fp32_out():
+    lens = syn.ragged_lengths(200, 100, 900, 6).tolist()
+    c = Case(L=3, w=2, Hq=32, Hkv=4, d=64, lens=lens, T_cap=910, seed=41, std=0.125, out_dtype=1)
+    _, _, stats = c.step()
+    # P is rounded to bf16 for the second MMA: errors stay far below the bf16-output bound
+    assert max(s[1] for s in stats) < 2e-3
+    c.step()
+    c.close()
+
+
+def test_mma_kernel_single_long_pair():
+    c = Case(L=2, w=0, Hq=8, Hkv=1, d=64, lens=[50000], T_cap=50010, seed=4, std=0.125)
+    c.step()
+    c.close()
+
+
+def test_tinyllama_shape_stack():
+    """22 layers, 32 q heads, 4 kv heads, d_h 64, w = 2, values scaled by 1/sqrt(d_h) (rel-L2 binds)."""
+    lens = [512, 513, 1024, 1535, 700, 511, 33, 1200]
+    c = Case(L=22, w=2, Hq=32, Hkv=4, d=64, lens=lens, T_cap=1540, seed=2, std=0.125)
+    c.step(); c.step()
+    c.close()
+
+
+def test_alu_kernel_forced_for_grouped_heads():
+    c = Case(L=3, w=2, Hq=16, Hkv=2, d=64, lens=[3, 64, 200, 511], T_cap=520, seed=8, std=0.125,
+             kernel_kind=1)
+    assert c.cache.info.kernel_kind == 1
+    c.step()
+    c.close()
