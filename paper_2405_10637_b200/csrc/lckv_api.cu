@@ -117,6 +117,11 @@ int resolve_kernel_kind(const lckv_config_t& c)
     return (c.kernel_kind == 0 && g % 8 == 0) ? 2 : 1;
 }
 
+int workers_per_sm(const lckv_config_t& c)
+{
+    return resolve_kernel_kind(c) == 2 ? lckv::kMmaWarps : lckv::kAluWarps;
+}
+
 int partial_record_floats(const lckv_config_t& c)
 {
     return resolve_kernel_kind(c) == 2 ? c.head_dim * 8 + 16 : c.head_dim + 4;
@@ -331,7 +336,7 @@ size_t lckv_cache_bytes(const lckv_config_t* cfg)
     int n_kv = 0;
     for (int l = 0; l < cfg->n_layers; ++l) n_kv += pl.write_slot[l] >= 0;
     Layout y;
-    make_layout(*cfg, pl.n_slots, sm * lckv::kAluWarps, n_kv, y);
+    make_layout(*cfg, pl.n_slots, sm * workers_per_sm(*cfg), n_kv, y);
     return y.total_bytes;
 }
 
@@ -350,7 +355,7 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     for (int l = 0; l < cfg->n_layers; ++l) c->n_kv_layers += c->plan.write_slot[l] >= 0;
     c->sm_count = sm;
     c->grid = sm;
-    c->n_workers = sm * lckv::kAluWarps;
+    c->n_workers = sm * workers_per_sm(*cfg);
     c->kernel_kind = resolve_kernel_kind(*cfg);
     c->rows_per_tile = lckv::kAluSlotBytes / (cfg->head_dim * 2);
     c->h_pairs = c->kernel_kind == 2 ? cfg->n_q_heads / 8 : cfg->n_q_heads;
@@ -576,7 +581,7 @@ int lckv_last_cuda_error(void) { return g_last_cuda_error; }
 // =============================================================================================
 namespace {
 
-constexpr int kStaticMaxWorkers = LCKV_STATIC_MAX_SMS * lckv::kAluWarps;
+constexpr int kStaticMaxWorkers = LCKV_STATIC_MAX_SMS * 8;  // worker records the scratch holds
 constexpr int kStaticPreStride = LCKV_STATIC_MAX_BATCH + 64;
 constexpr size_t kStOffPre = 0;
 constexpr size_t kStOffStart = kStOffPre + 2 * (size_t)kStaticPreStride * 4;
@@ -639,10 +644,10 @@ extern "C" int lckv_decode_attention_static(const void* k, const void* v, const 
     if (!g_static_ptr[dev])
         if (int rc = static_setup(dev)) return rc;
     const int sms = g_static_sms[dev];
-    if (sms > LCKV_STATIC_MAX_SMS) return LCKV_ESTATICLIMIT;
+    const int n_workers = sms * lckv::kAluWarps;
+    if (sms > LCKV_STATIC_MAX_SMS || n_workers > kStaticMaxWorkers) return LCKV_ESTATICLIMIT;
     unsigned char* base = g_static_ptr[dev];
     cudaStream_t st = static_cast<cudaStream_t>(stream);
-    const int n_workers = sms * lckv::kAluWarps;
     uint32_t* d_pre = reinterpret_cast<uint32_t*>(base + kStOffPre);
     int32_t* d_start = reinterpret_cast<int32_t*>(base + kStOffStart);
     int32_t* d_counters = reinterpret_cast<int32_t*>(base + kStOffCounters);

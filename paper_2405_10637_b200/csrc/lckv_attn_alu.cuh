@@ -19,8 +19,18 @@
 
 namespace lckv {
 
-constexpr int kAluWarps = 8;         // workers per CTA
-constexpr int kAluSlots = 6;         // ring slots per worker
+// Tuning knobs (compile-time): workers per CTA, ring slots per worker, packed fp32x2 FMAs.
+#ifndef LCKV_ALU_WARPS
+#define LCKV_ALU_WARPS 8
+#endif
+#ifndef LCKV_ALU_SLOTS
+#define LCKV_ALU_SLOTS 4
+#endif
+#ifndef LCKV_ALU_FFMA2
+#define LCKV_ALU_FFMA2 1
+#endif
+constexpr int kAluWarps = LCKV_ALU_WARPS;  // workers per CTA
+constexpr int kAluSlots = LCKV_ALU_SLOTS;  // ring slots per worker
 constexpr int kAluSlotBytes = 4096;  // one tile of K or of V
 constexpr int kAluSmemBytes = kAluWarps * kAluSlots * (kAluSlotBytes + 8);
 
@@ -151,6 +161,12 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
     bool ok = true;
 
     float qf[8];
+#if LCKV_ALU_FFMA2
+    uint64_t q2[4];   // the same eight values as fp32 pairs
+    uint64_t o2[4];   // output accumulators as fp32 pairs (o[] is filled from them at the end)
+#pragma unroll
+    for (int j = 0; j < 4; ++j) o2[j] = 0ull;
+#endif
     auto load_q = [&](const TileCursor& c) {
         const uint4 raw =
             __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)c.b * H + c.h) * D) + a);
@@ -158,6 +174,10 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
         qf[2] = bf16lo(raw.y) * p.scale_log2; qf[3] = bf16hi(raw.y) * p.scale_log2;
         qf[4] = bf16lo(raw.z) * p.scale_log2; qf[5] = bf16hi(raw.z) * p.scale_log2;
         qf[6] = bf16lo(raw.w) * p.scale_log2; qf[7] = bf16hi(raw.w) * p.scale_log2;
+#if LCKV_ALU_FFMA2
+#pragma unroll
+        for (int j = 0; j < 4; ++j) q2[j] = pack_f32x2(qf[2 * j], qf[2 * j + 1]);
+#endif
     };
     load_q(cc);
     uint32_t seg_t0 = cc.t;
@@ -177,6 +197,15 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
 #pragma unroll
             for (int i = 0; i < NP; ++i) {
                 const uint4 kv = lds128(base + i * (RPI * D * 2));
+#if LCKV_ALU_FFMA2
+                uint64_t acc = fmul2(pack_f32x2(bf16lo(kv.x), bf16hi(kv.x)), q2[0]);
+                acc = ffma2(pack_f32x2(bf16lo(kv.y), bf16hi(kv.y)), q2[1], acc);
+                acc = ffma2(pack_f32x2(bf16lo(kv.z), bf16hi(kv.z)), q2[2], acc);
+                acc = ffma2(pack_f32x2(bf16lo(kv.w), bf16hi(kv.w)), q2[3], acc);
+                float ax, ay;
+                unpack_f32x2(acc, ax, ay);
+                part[i] = ax + ay;
+#else
                 float s = bf16lo(kv.x) * qf[0];
                 s = fmaf(bf16hi(kv.x), qf[1], s);
                 s = fmaf(bf16lo(kv.y), qf[2], s);
@@ -186,6 +215,7 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
                 s = fmaf(bf16lo(kv.w), qf[6], s);
                 s = fmaf(bf16hi(kv.w), qf[7], s);
                 part[i] = s;
+#endif
             }
         }
         __syncwarp();
@@ -231,8 +261,16 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
         const float pr = ex2(s - m_new);
         l_run = fmaf(l_run, alpha, pr);
         m_run = m_new;
+#if LCKV_ALU_FFMA2
+        {
+            const uint64_t a2 = pack_f32x2(alpha, alpha);
+#pragma unroll
+            for (int j = 0; j < 4; ++j) o2[j] = fmul2(o2[j], a2);
+        }
+#else
 #pragma unroll
         for (int k = 0; k < 8; ++k) o[k] *= alpha;
+#endif
 
         // ---- V tile: weighted sum -----------------------------------------------------------
         if (!mbar_wait_bounded(bars + 8 * cslot, cphase)) { ok = false; break; }
@@ -251,6 +289,13 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
             for (int i = 0; i < NP; ++i) {
                 const float pi = __shfl_sync(FULL, pr, grp * LPR + i * DUP);
                 const uint4 vv = lds128(base + i * (RPI * D * 2));
+#if LCKV_ALU_FFMA2
+                const uint64_t p2 = pack_f32x2(pi, pi);
+                o2[0] = ffma2(p2, pack_f32x2(bf16lo(vv.x), bf16hi(vv.x)), o2[0]);
+                o2[1] = ffma2(p2, pack_f32x2(bf16lo(vv.y), bf16hi(vv.y)), o2[1]);
+                o2[2] = ffma2(p2, pack_f32x2(bf16lo(vv.z), bf16hi(vv.z)), o2[2]);
+                o2[3] = ffma2(p2, pack_f32x2(bf16lo(vv.w), bf16hi(vv.w)), o2[3]);
+#else
                 o[0] = fmaf(pi, bf16lo(vv.x), o[0]);
                 o[1] = fmaf(pi, bf16hi(vv.x), o[1]);
                 o[2] = fmaf(pi, bf16lo(vv.y), o[2]);
@@ -259,6 +304,7 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
                 o[5] = fmaf(pi, bf16hi(vv.z), o[5]);
                 o[6] = fmaf(pi, bf16lo(vv.w), o[6]);
                 o[7] = fmaf(pi, bf16hi(vv.w), o[7]);
+#endif
             }
         }
         __syncwarp();
@@ -271,6 +317,10 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
         const bool last = (tile + 1 == n_tiles);
         if (pair_end || last) {
             // everything this worker saw of the pair: reduce over row groups and lanes
+#if LCKV_ALU_FFMA2
+#pragma unroll
+            for (int j = 0; j < 4; ++j) unpack_f32x2(o2[j], o[2 * j], o[2 * j + 1]);
+#endif
 #pragma unroll
             for (int off = LPR; off < 32; off <<= 1)
 #pragma unroll
@@ -304,23 +354,28 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
                 ticket = __shfl_sync(FULL, ticket, 0);
                 if (ticket == (int)(c_last - c_first)) {
                     // Last contributor: merge every part in worker order (fixed summation order).
+                    // Record addresses do not depend on loaded data, so the unrolled loops keep
+                    // several L2 round trips in flight.
                     __threadfence();
+                    const uint64_t lo_first = (uint64_t)c_first * total / n_eff;
+                    const float* rec0 = p.partials + (size_t)(2 * c_first) * REC;
+                    const int first_odd = (gs != lo_first) ? 1 : 0;  // which record of c_first
+                    const int n_parts = (int)(c_last - c_first) + 1;
                     float M = -INFINITY;
-                    for (uint32_t c = c_first; c <= c_last; ++c) {
-                        const uint64_t lo_c = (uint64_t)c * total / n_eff;
-                        const float* r = p.partials +
-                            (size_t)(2 * c + ((c == c_first && gs != lo_c) ? 1 : 0)) * REC;
+#pragma unroll 4
+                    for (int i = 0; i < n_parts; ++i) {
+                        const float* r = rec0 + (size_t)(2 * i + (i == 0 ? first_odd : 0)) * REC;
                         M = fmaxf(M, __ldcg(r + D));
                     }
                     float Lsum = 0.f, acc[8];
 #pragma unroll
                     for (int k = 0; k < 8; ++k) acc[k] = 0.f;
-                    for (uint32_t c = c_first; c <= c_last; ++c) {
-                        const uint64_t lo_c = (uint64_t)c * total / n_eff;
-                        const float* r = p.partials +
-                            (size_t)(2 * c + ((c == c_first && gs != lo_c) ? 1 : 0)) * REC;
-                        const float wgt = ex2(__ldcg(r + D) - M);
-                        Lsum = fmaf(__ldcg(r + D + 1), wgt, Lsum);
+#pragma unroll 4
+                    for (int i = 0; i < n_parts; ++i) {
+                        const float* r = rec0 + (size_t)(2 * i + (i == 0 ? first_odd : 0)) * REC;
+                        const float2 ml = __ldcg(reinterpret_cast<const float2*>(r + D));
+                        const float wgt = ex2(ml.x - M);
+                        Lsum = fmaf(ml.y, wgt, Lsum);
                         if (lane < LPR) {
                             const float4 x0 = __ldcg(reinterpret_cast<const float4*>(r) + 2 * lane);
                             const float4 x1 =
@@ -364,6 +419,10 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
             l_run = 0.f;
 #pragma unroll
             for (int k = 0; k < 8; ++k) o[k] = 0.f;
+#if LCKV_ALU_FFMA2
+#pragma unroll
+            for (int j = 0; j < 4; ++j) o2[j] = 0ull;
+#endif
         }
         if (!last) {
             cursor_next(cc, p, H);

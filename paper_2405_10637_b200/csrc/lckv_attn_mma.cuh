@@ -17,8 +17,14 @@
 
 namespace lckv {
 
-constexpr int kMmaWarps = 8;
-constexpr int kMmaSlots = 6;
+#ifndef LCKV_MMA_WARPS
+#define LCKV_MMA_WARPS 8
+#endif
+#ifndef LCKV_MMA_SLOTS
+#define LCKV_MMA_SLOTS 3
+#endif
+constexpr int kMmaWarps = LCKV_MMA_WARPS;
+constexpr int kMmaSlots = LCKV_MMA_SLOTS;
 constexpr int kMmaSlotBytes = 4096;
 constexpr int kMmaSmemBytes = kMmaWarps * kMmaSlots * (kMmaSlotBytes + 8) + 1024;  // + alignment slack
 
@@ -63,6 +69,48 @@ __device__ __forceinline__ uint32_t cvt_bf16x2(float lo, float hi)
     uint32_t d;
     asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(d) : "f"(hi), "f"(lo));
     return d;
+}
+
+// Position in a launch's tile sequence, with everything a copy needs kept incrementally (no
+// division or 64-bit multiply per tile).
+struct RowCursor {
+    int32_t b, h;      // sequence; pair within the sequence
+    uint32_t t, nt;    // tile within the pair; tiles per pair of sequence b
+    int32_t nv;        // visible rows of sequence b
+    int32_t kvh, sub;  // kv head the pair reads; index of the pair among the pairs of that kv head
+    int64_t row;       // cache row (of the [B*H_kv*T_cap, D] view) where the tile starts
+};
+
+__device__ __forceinline__ void rcursor_load(RowCursor& c, const AttnParams& p)
+{
+    c.nt = __ldg(p.pre + c.b + 1) - __ldg(p.pre + c.b);
+    c.nv = __ldg(p.lens + c.b) + p.mode;
+}
+
+// After b, h, t are set: derive the kv head and the tile's first row.  per_kv = pairs per kv head.
+__device__ __forceinline__ void rcursor_seek(RowCursor& c, const AttnParams& p, int per_kv, int R)
+{
+    c.kvh = c.h / per_kv;
+    c.sub = c.h - c.kvh * per_kv;
+    c.row = ((int64_t)c.b * p.H_kv + c.kvh) * p.T_cap + (int64_t)c.t * R;
+}
+
+// Next tile in (b, pair, tile) order, skipping sequences without tiles.  Safe past the end.
+__device__ __forceinline__ void rcursor_next(RowCursor& c, const AttnParams& p, int H, int per_kv,
+                                            int R)
+{
+    if (++c.t < c.nt) { c.row += R; return; }
+    c.t = 0;
+    if (++c.h < H) {
+        if (++c.sub == per_kv) { c.sub = 0; ++c.kvh; }
+    } else {
+        c.h = 0; c.sub = 0; c.kvh = 0;
+        do {
+            if (++c.b >= p.B) { c.b = p.B; c.nt = 0; c.nv = 0; return; }
+            rcursor_load(c, p);
+        } while (c.nt == 0);
+    }
+    c.row = ((int64_t)c.b * p.H_kv + c.kvh) * p.T_cap;
 }
 
 struct MmaParams {
@@ -125,20 +173,20 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
     const uint32_t n_tiles = (uint32_t)(hi - lo);
     const uint32_t n_items = 2 * n_tiles;
 
-    TileCursor cc;
+    RowCursor cc;
     cc.b = __ldg(p.start_b + w);
-    cursor_load(cc, p);
+    rcursor_load(cc, p);
     {
         const uint64_t rel = lo - (uint64_t)__ldg(p.pre + cc.b) * (uint64_t)H;
         cc.h = (int32_t)(rel / cc.nt);
         cc.t = (uint32_t)(rel % cc.nt);
     }
-    TileCursor ci = cc;
+    rcursor_seek(cc, p, mp.groups_per_kv, R);
+    RowCursor ci = cc;
 
     uint32_t issued = 0, islot = 0;
     auto issue = [&]() {
-        const int kvh = ci.h / mp.groups_per_kv;
-        const int64_t row = ((int64_t)ci.b * p.H_kv + kvh) * p.T_cap + (int64_t)ci.t * R;
+        const int64_t row = ci.row;
         if (lane == 0) {
             const void* tm = (issued & 1) ? (const void*)&tmV : (const void*)&tmK;
             mbar_expect_tx(bars + 8 * islot, kMmaSlotBytes);
@@ -147,7 +195,7 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
                 tma_load_2d(ring + islot * kMmaSlotBytes + bx * BOX_BYTES, tm, bx * 64, (int32_t)row,
                             bars + 8 * islot);
         }
-        if (issued & 1) cursor_next(ci, p, H);
+        if (issued & 1) rcursor_next(ci, p, H, mp.groups_per_kv, R);
         ++issued;
         islot = (islot + 1 == NS) ? 0 : islot + 1;
     };
@@ -161,7 +209,7 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
 
     // Q^T fragments of the pair's 8 query heads: lane holds query g4, dims 2*c4 (+1) (+8) per k-step.
     uint32_t qb[KS][2];
-    auto load_q = [&](const TileCursor& c) {
+    auto load_q = [&](const RowCursor& c) {
         const uint16_t* qp = p.q + ((size_t)c.b * mp.n_q_heads + (size_t)c.h * 8 + g4) * D + 2 * c4;
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
@@ -320,13 +368,17 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
                 ticket = __shfl_sync(FULL, ticket, 0);
                 if (ticket == (int)(c_last - c_first)) {
                     __threadfence();
+                    const uint64_t lo_first = (uint64_t)c_first * total / n_eff;
+                    const float* rec0 = p.partials + (size_t)(2 * c_first) * REC;
+                    const int first_odd = (gs != lo_first) ? 1 : 0;
+                    const int n_parts = (int)(c_last - c_first) + 1;
                     float M[2] = {-INFINITY, -INFINITY};
-                    for (uint32_t c = c_first; c <= c_last; ++c) {
-                        const uint64_t lo_c = (uint64_t)c * total / n_eff;
-                        const float* r = p.partials +
-                            (size_t)(2 * c + ((c == c_first && gs != lo_c) ? 1 : 0)) * REC;
-                        M[0] = fmaxf(M[0], __ldcg(r + D * 8 + 2 * c4));
-                        M[1] = fmaxf(M[1], __ldcg(r + D * 8 + 2 * c4 + 1));
+#pragma unroll 4
+                    for (int i = 0; i < n_parts; ++i) {
+                        const float* r = rec0 + (size_t)(2 * i + (i == 0 ? first_odd : 0)) * REC;
+                        const float2 mm = __ldcg(reinterpret_cast<const float2*>(r + D * 8) + c4);
+                        M[0] = fmaxf(M[0], mm.x);
+                        M[1] = fmaxf(M[1], mm.y);
                     }
                     float Ls[2] = {0.f, 0.f};
                     float acc[MT][4];
@@ -334,14 +386,15 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
                     for (int mt = 0; mt < MT; ++mt)
 #pragma unroll
                         for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
-                    for (uint32_t c = c_first; c <= c_last; ++c) {
-                        const uint64_t lo_c = (uint64_t)c * total / n_eff;
-                        const float* r = p.partials +
-                            (size_t)(2 * c + ((c == c_first && gs != lo_c) ? 1 : 0)) * REC;
-                        const float w0 = ex2(__ldcg(r + D * 8 + 2 * c4) - M[0]);
-                        const float w1 = ex2(__ldcg(r + D * 8 + 2 * c4 + 1) - M[1]);
-                        Ls[0] = fmaf(__ldcg(r + D * 8 + 8 + 2 * c4), w0, Ls[0]);
-                        Ls[1] = fmaf(__ldcg(r + D * 8 + 8 + 2 * c4 + 1), w1, Ls[1]);
+#pragma unroll 2
+                    for (int i = 0; i < n_parts; ++i) {
+                        const float* r = rec0 + (size_t)(2 * i + (i == 0 ? first_odd : 0)) * REC;
+                        const float2 mm = __ldcg(reinterpret_cast<const float2*>(r + D * 8) + c4);
+                        const float2 ll = __ldcg(reinterpret_cast<const float2*>(r + D * 8 + 8) + c4);
+                        const float w0 = ex2(mm.x - M[0]);
+                        const float w1 = ex2(mm.y - M[1]);
+                        Ls[0] = fmaf(ll.x, w0, Ls[0]);
+                        Ls[1] = fmaf(ll.y, w1, Ls[1]);
 #pragma unroll
                         for (int mt = 0; mt < MT; ++mt) {
                             const float4 x = __ldcg(reinterpret_cast<const float4*>(r) + mt * 32 + lane);
@@ -399,7 +452,7 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
                 for (int i = 0; i < 4; ++i) o[mt][i] = 0.f;
         }
         if (!last) {
-            cursor_next(cc, p, H);
+            rcursor_next(cc, p, H, mp.groups_per_kv, R);
             if (pair_end) { load_q(cc); seg_t0 = 0; }
         }
     }
