@@ -225,11 +225,10 @@ def run_ours(args):
     local = int(os.environ.get("LOCAL_RANK", "0"))
     if world != args.gpus and world > 1:
         raise SystemExit("--gpus must equal WORLD_SIZE under torchrun")
-    dist = None
+    from paper_2405_10637_b200 import multi
+    torch.cuda.set_device(local)
     if world > 1:
-        import torch.distributed as dist_
-        dist = dist_
-        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+        multi.init("nccl", torch.device(f"cuda:{local}"))
     torch.cuda.set_device(local)
     dev = torch.device(f"cuda:{local}")
     stream = torch.cuda.current_stream()
@@ -281,16 +280,11 @@ def run_ours(args):
 
     def barrier():
         torch.cuda.synchronize()
-        if dist:
-            dist.barrier()
+        multi.barrier()
         torch.cuda.synchronize()
 
     def max_over_ranks(ms):
-        if not dist:
-            return ms
-        t = torch.tensor([ms], device=dev, dtype=torch.float64)
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-        return float(t.item())
+        return multi.max_over_ranks(ms, dev)
 
     # ---- headline: K steps at the full batch --------------------------------------------------
     step = make_step(B)
@@ -383,7 +377,8 @@ def run_ours(args):
             "roofline": roofline, "cpu_baseline": cpu, "sweep": sweep,
         }))
     cache.close()
-    if dist:
+    if world > 1:
+        import torch.distributed as dist
         dist.destroy_process_group()
 
 

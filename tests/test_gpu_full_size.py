@@ -1,0 +1,105 @@
+"""Parity at the full benchmark sizes, in the launch configuration bench.py times.
+
+The oracle cannot run a whole 0.5 TB step, so it checks sampled output rows one by one: for a
+sampled (layer, sequence, head) the visible K/V rows and the query are copied from the device and
+attended on the CPU in float64.  On top of that: every output finite, lengths advanced by exactly
+one, appended rows bit-identical to the step's k/v.  Inputs are the bench's (seeded, device-drawn).
+"""
+import numpy as np
+import pytest
+import torch
+
+from oracle import lckv_oracle as orc
+from paper_2405_10637_b200 import binding as lk
+from paper_2405_10637_b200 import inputs as syn
+from helpers import MAX_ABS, REL_L2
+
+pytestmark = pytest.mark.gpu
+
+
+def run_full(wl, B, lens, T_cap, n_samples, seed, top_variant=0, steps=1):
+    L, Hq, Hkv, d = wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
+    g = Hq // Hkv
+    cfg = lk.make_config(L, wl.n_warmup, Hq, Hkv, d, B, T_cap, top_variant=top_variant)
+    cache = lk.Cache(cfg)
+    dev = cache.device
+    plan = lk.lckv_plan(L, wl.n_warmup, top_variant)
+    for s in range(cache.info.n_slots):
+        kt, vt = cache.slot_tensors(s)
+        syn.fill_randn_bf16_(kt, syn.seed_for(wl, syn.T_K, s), std=wl.std)
+        syn.fill_randn_bf16_(vt, syn.seed_for(wl, syn.T_V, s), std=wl.std)
+    cache.lckv_cache_reset(lens.tolist())
+    rng = np.random.default_rng(seed)
+    scale = d ** -0.5
+    cur = lens.astype(np.int64).copy()
+    for step in range(steps):
+        q = [syn.randn_bf16((B, Hq, d), 900 + l + 100 * step, device=dev, std=wl.std) for l in range(L)]
+        kv = [syn.randn_bf16((B, Hkv, d), 950 + l + 100 * step, device=dev, std=wl.std)
+              if plan["write_slot"][l] >= 0 else None for l in range(L)]
+        outs = [torch.full((B, Hq, d), float("nan"), dtype=torch.bfloat16, device=dev) for _ in range(L)]
+        cache.lckv_layer_stack_step(q, outs, kv, kv)
+        torch.cuda.synchronize()
+        assert cache.lckv_cache_status() == 0
+        for l in range(L):
+            assert torch.isfinite(outs[l].float()).all(), f"layer {l}: non-finite output"
+        errs, refs = [], []
+        for _ in range(n_samples):
+            l, b, h = int(rng.integers(L)), int(rng.integers(B)), int(rng.integers(Hq))
+            slot, mode = plan["read_slot"][l], plan["mode"][l]
+            n_vis = int(cur[b]) + mode
+            kt, vt = cache.slot_tensors(slot)
+            o, _ = orc.attend_row(syn.bits(q[l][b, h]), syn.bits(kt[b, h // g, :n_vis]),
+                                  syn.bits(vt[b, h // g, :n_vis]), scale)
+            got = outs[l][b, h].float().cpu().numpy().astype(np.float64)
+            assert np.abs(got - o).max() <= MAX_ABS, (l, b, h, np.abs(got - o).max())
+            errs.append(got - o); refs.append(o)
+        rel = np.linalg.norm(np.stack(errs)) / np.linalg.norm(np.stack(refs))
+        assert rel <= REL_L2, rel
+        # appended rows and lengths (bit-exact), on a few sequences
+        for l in range(L):
+            if plan["write_slot"][l] < 0:
+                continue
+            kt, vt = cache.slot_tensors(plan["write_slot"][l])
+            for b in rng.integers(B, size=3):
+                row = int(cur[b])
+                assert torch.equal(kt[b, :, row], kv[l][b]) and torch.equal(vt[b, :, row], kv[l][b])
+        cur += 1
+        assert cache.lckv_cache_lengths(B) == cur.tolist()
+    cache.close()
+
+
+def test_llama7b_ragged_batch_512():
+    """Llama-7B shape, w = 2, ragged lengths uniform in [256, 4096], B = 512 (the headline case)."""
+    wl = syn.WORKLOADS["llama7b"]
+    B = 512
+    lens = syn.ragged_lengths(B, 256, 4096, syn.seed_for(wl, syn.T_LENS)).numpy()
+    run_full(wl, B, lens, 4096 + 64, n_samples=48, seed=1)
+
+
+def test_llama7b_small_batch_8_variant1():
+    """The small end of the batch sweep (every pair split over several workers), reading 2 of 'top layer'."""
+    wl = syn.WORKLOADS["llama7b"]
+    lens = syn.ragged_lengths(8, 256, 4096, syn.seed_for(wl, syn.T_LENS)).numpy()
+    run_full(wl, 8, lens, 4096 + 64, n_samples=48, seed=2, top_variant=1, steps=2)
+
+
+def test_tinyllama_batch_128_decode_steps():
+    """TinyLlama shape (GQA 8:1), B = 128, prompt 512, three decode steps."""
+    wl = syn.WORKLOADS["tinyllama"]
+    lens = np.full(128, 512, np.int32)
+    run_full(wl, 128, lens, 1536, n_samples=48, seed=3, steps=3)
+
+
+def test_llama30b_batch_256():
+    """Llama-30B shape: 60 layers, 52 heads (not a power of two), context 2048, B = 256."""
+    wl = syn.WORKLOADS["llama30b"]
+    lens = np.full(256, 2048, np.int32)
+    run_full(wl, 256, lens, 2048 + 64, n_samples=32, seed=4)
+
+
+@pytest.mark.parametrize("w,B,T", [(0, 64, 8192), (8, 64, 8192), (2, 8, 32768)])
+def test_long_context_warmup_sweep(w, B, T):
+    """7B shape at long context for several warmup counts (footprint max(w,1) caches)."""
+    wl = syn.WORKLOADS["sweep7b"].with_(n_warmup=w)
+    lens = np.full(B, T, np.int32)
+    run_full(wl, B, lens, T + 64, n_samples=24, seed=5 + w)
