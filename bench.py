@@ -231,6 +231,7 @@ def run_ours(args):
         multi.init("nccl", torch.device(f"cuda:{local}"))
     torch.cuda.set_device(local)
     dev = torch.device(f"cuda:{local}")
+    torch.cuda.set_stream(torch.cuda.Stream(device=dev))  # a capturable (non-default) stream
     stream = torch.cuda.current_stream()
 
     wl, p = workload_params(args)

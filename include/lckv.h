@@ -69,7 +69,8 @@ typedef struct {
     int32_t out_dtype;     /* 0 = bf16 outputs, 1 = fp32 outputs                             */
     int32_t host_staging;  /* 1: reserve device staging for lckv_layer_stack_step_host       */
     int32_t use_graph;     /* 1: lckv_layer_stack_step replays a CUDA graph when the argument
-                              pointers repeat from the previous call                         */
+                              pointers repeat from the previous call (needs a stream other
+                              than the legacy default stream; otherwise plain launches)      */
     int32_t kernel_kind;   /* 0 = choose (tensor-core kernel when the query group is a dense
                               MMA tile, else the FP32-ALU kernel); 1 = force FP32-ALU        */
 } lckv_config_t;

@@ -88,6 +88,11 @@ struct lckv_cache {
     std::vector<int32_t> h_lens;  // host mirror of the device lengths
     int n_kv_layers;
     std::vector<CUtensorMap> tm_k, tm_v;  // per slot, tensor-core kernel only
+    int ws_parity;                        // which half of the split-K workspace the next launch uses
+    size_t partials_half_floats;          // floats in one half of the partial records
+    // CUDA graph of one step, valid for the argument pointers it was captured with
+    cudaGraphExec_t graph_exec;
+    std::vector<const void*> graph_key;
 };
 
 namespace {
@@ -167,10 +172,10 @@ void make_layout(const lckv_config_t& c, int n_slots, int n_workers, int n_kv_la
     y.pre_stride = (int)align_up((size_t)c.max_batch + 1, 64);
     y.off_pre = off;       off = align_up(off + 2 * (size_t)y.pre_stride * 4, A);
     y.off_start = off;     off = align_up(off + 2 * (size_t)n_workers * 4, A);
-    y.off_counters = off;  off = align_up(off + (size_t)n_workers * 4, A);
+    y.off_counters = off;  off = align_up(off + 2 * (size_t)n_workers * 4, A);  // two halves
     y.off_status = off;    off = align_up(off + 4, A);
     y.off_partials = off;
-    off = align_up(off + 2 * (size_t)n_workers * partial_record_floats(c) * 4, A);
+    off = align_up(off + 2 * 2 * (size_t)n_workers * partial_record_floats(c) * 4, A);  // two halves
     y.workspace_bytes = off;
     y.slot_bytes =
         align_up((size_t)c.max_batch * c.n_kv_heads * (size_t)c.max_seq * c.head_dim * 2, A);
@@ -220,8 +225,29 @@ int launch_plan(lckv_cache* c, int batch, cudaStream_t st)
     return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
 }
 
+// Launch with the programmatic-serialization attribute: the kernel may be scheduled while its
+// predecessor in the stream drains; it orders itself with griddepcontrol.wait.
+template <typename... KArgs, typename... Args>
+cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, size_t smem, cudaStream_t st,
+                       Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(block);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+// early: the previous kernel in the stream is an attention launch of the same step and this one
+// reads only rows that were final before it (condensed mode), so its first copies need not wait.
 int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out, float* lse,
-                     int batch, cudaStream_t st)
+                     int batch, cudaStream_t st, bool early = false)
 {
     lckv::AttnParams p;
     p.K = slot_k(c, slot);
@@ -232,8 +258,10 @@ int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out
     p.lens = c->d_lens;
     p.pre = c->d_pre + (size_t)mode * c->lay.pre_stride;
     p.start_b = c->d_start + (size_t)mode * c->n_workers;
-    p.partials = c->d_partials;
-    p.counters = c->d_counters;
+    // consecutive launches may overlap at their edges: alternate the split-K workspace halves
+    p.partials = c->d_partials + (size_t)c->ws_parity * c->partials_half_floats;
+    p.counters = c->d_counters + (size_t)c->ws_parity * c->n_workers;
+    c->ws_parity ^= 1;
     p.status = c->d_status;
     p.T_cap = c->cfg.max_seq;
     p.B = batch;
@@ -243,6 +271,8 @@ int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out
     p.n_workers = c->n_workers;
     p.out_f32 = c->cfg.out_dtype;
     p.scale_log2 = c->scale_log2;
+    p.early_kv = early ? 1 : 0;
+    cudaError_t e;
     if (c->kernel_kind == 2) {
         lckv::MmaParams mp;
         mp.a = p;
@@ -250,17 +280,19 @@ int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out
         mp.n_q_heads = c->cfg.n_q_heads;
         mp.groups_per_kv = c->cfg.n_q_heads / c->cfg.n_kv_heads / 8;
         if (c->cfg.head_dim == 128)
-            lckv::attn_mma_kernel<128><<<c->grid, lckv::kMmaWarps * 32, lckv::kMmaSmemBytes, st>>>(
-                mp, c->tm_k[slot], c->tm_v[slot]);
+            e = launch_pdl(lckv::attn_mma_kernel<128>, c->grid, lckv::kMmaWarps * 32,
+                           lckv::kMmaSmemBytes, st, mp, c->tm_k[slot], c->tm_v[slot]);
         else
-            lckv::attn_mma_kernel<64><<<c->grid, lckv::kMmaWarps * 32, lckv::kMmaSmemBytes, st>>>(
-                mp, c->tm_k[slot], c->tm_v[slot]);
+            e = launch_pdl(lckv::attn_mma_kernel<64>, c->grid, lckv::kMmaWarps * 32,
+                           lckv::kMmaSmemBytes, st, mp, c->tm_k[slot], c->tm_v[slot]);
     } else if (c->cfg.head_dim == 128) {
-        lckv::attn_alu_kernel<128><<<c->grid, lckv::kAluWarps * 32, lckv::kAluSmemBytes, st>>>(p);
+        e = launch_pdl(lckv::attn_alu_kernel<128>, c->grid, lckv::kAluWarps * 32,
+                       lckv::kAluSmemBytes, st, p);
     } else {
-        lckv::attn_alu_kernel<64><<<c->grid, lckv::kAluWarps * 32, lckv::kAluSmemBytes, st>>>(p);
+        e = launch_pdl(lckv::attn_alu_kernel<64>, c->grid, lckv::kAluWarps * 32,
+                       lckv::kAluSmemBytes, st, p);
     }
-    return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
+    return cuda_ok(e) ? LCKV_OK : LCKV_ECUDA;
 }
 
 int launch_append(lckv_cache* c, int slot, const void* k_new, const void* v_new, int batch,
@@ -279,9 +311,12 @@ int launch_append(lckv_cache* c, int slot, const void* k_new, const void* v_new,
 int launch_advance(lckv_cache* c, int batch, cudaStream_t st)
 {
     lckv::advance_kernel<<<(batch + 255) / 256, 256, 0, st>>>(c->d_lens, batch);
-    if (!cuda_ok(cudaGetLastError())) return LCKV_ECUDA;
+    return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
+}
+
+void mirror_advance(lckv_cache* c, int batch)
+{
     for (int b = 0; b < batch; ++b) c->h_lens[b] += 1;
-    return LCKV_OK;
 }
 
 // The launches of one step, in the order the header states.
@@ -290,17 +325,86 @@ int enqueue_step(lckv_cache* c, const void* const* q, void* const* out, const vo
 {
     const Plan& pl = c->plan;
     const int L = c->cfg.n_layers;
+    // A step starts after fully serialised launches (advance, plan), so it may always begin with
+    // workspace half 0; this also makes a captured step replayable.
+    c->ws_parity = 0;
     if (int rc = launch_plan(c, batch, st)) return rc;
+    bool prev_attn = false;
     for (int l = 0; l < L; ++l) {
-        if (pl.write_slot[l] >= 0 && pl.write_before[l])
+        if (pl.write_slot[l] >= 0 && pl.write_before[l]) {
             if (int rc = launch_append(c, pl.write_slot[l], kn[l], vn[l], batch, st)) return rc;
-        if (int rc = launch_attention(c, pl.read_slot[l], pl.mode[l], q[l], out[l], nullptr, batch, st))
+            prev_attn = false;
+        }
+        const bool early = prev_attn && pl.mode[l] == LCKV_MODE_CONDENSED;
+        if (int rc = launch_attention(c, pl.read_slot[l], pl.mode[l], q[l], out[l], nullptr, batch,
+                                      st, early))
             return rc;
+        prev_attn = true;
     }
     for (int l = 0; l < L; ++l)
         if (pl.write_slot[l] >= 0 && !pl.write_before[l])
             if (int rc = launch_append(c, pl.write_slot[l], kn[l], vn[l], batch, st)) return rc;
     return launch_advance(c, batch, st);
+}
+
+void drop_graph(lckv_cache* c)
+{
+    if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
+    c->graph_exec = nullptr;
+    c->graph_key.clear();
+}
+
+// One step through a CUDA graph that is re-captured whenever the argument pointers, the batch or
+// the workspace parity differ from the captured ones.
+int step_with_graph(lckv_cache* c, const void* const* q, void* const* out, const void* const* kn,
+                    const void* const* vn, int batch, cudaStream_t st)
+{
+    const int L = c->cfg.n_layers;
+    std::vector<const void*> key;
+    key.reserve(4 * L + 1);
+    key.push_back(reinterpret_cast<const void*>((uintptr_t)batch));
+    for (int l = 0; l < L; ++l) {
+        key.push_back(q[l]);
+        key.push_back(out[l]);
+        key.push_back(c->plan.write_slot[l] >= 0 ? kn[l] : nullptr);
+        key.push_back(c->plan.write_slot[l] >= 0 ? vn[l] : nullptr);
+    }
+    if (!c->graph_exec || key != c->graph_key) {
+        drop_graph(c);
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (!cuda_ok(cudaStreamIsCapturing(st, &cs))) return LCKV_ECUDA;
+        // The caller is capturing already, or the stream is the legacy default stream (which
+        // cannot be captured): just issue the launches.
+        if (cs != cudaStreamCaptureStatusNone || st == nullptr || st == cudaStreamLegacy)
+            return enqueue_step(c, q, out, kn, vn, batch, st);
+        if (cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal) != cudaSuccess) {
+            (void)cudaGetLastError();
+            return enqueue_step(c, q, out, kn, vn, batch, st);
+        }
+        const int rc = enqueue_step(c, q, out, kn, vn, batch, st);
+        cudaGraph_t g = nullptr;
+        const bool ended = cuda_ok(cudaStreamEndCapture(st, &g));
+        if (rc || !ended || !g) {
+            if (g) cudaGraphDestroy(g);
+            return rc ? rc : LCKV_ECUDA;
+        }
+        const bool inst = cuda_ok(cudaGraphInstantiate(&c->graph_exec, g, 0));
+        cudaGraphDestroy(g);
+        if (!inst) { c->graph_exec = nullptr; return LCKV_ECUDA; }
+        c->graph_key = key;
+    }
+    if (!cuda_ok(cudaGraphLaunch(c->graph_exec, st))) return LCKV_ECUDA;
+    c->ws_parity = c->cfg.n_layers & 1;  // where the captured step leaves it
+    return LCKV_OK;
+}
+
+int run_step(lckv_cache* c, const void* const* q, void* const* out, const void* const* kn,
+             const void* const* vn, int batch, cudaStream_t st)
+{
+    const int rc = c->cfg.use_graph ? step_with_graph(c, q, out, kn, vn, batch, st)
+                                    : enqueue_step(c, q, out, kn, vn, batch, st);
+    if (rc == LCKV_OK) mirror_advance(c, batch);
+    return rc;
 }
 
 }  // namespace
@@ -372,6 +476,9 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     c->d_status = reinterpret_cast<int32_t*>(c->base + c->lay.off_status);
     c->d_partials = reinterpret_cast<float*>(c->base + c->lay.off_partials);
     c->h_lens.assign(cfg->max_batch, 0);
+    c->ws_parity = 0;
+    c->partials_half_floats = 2 * (size_t)c->n_workers * partial_record_floats(*cfg);
+    c->graph_exec = nullptr;
 
     if (c->kernel_kind == 2) {
         const uint64_t rows = (uint64_t)cfg->max_batch * cfg->n_kv_heads * (uint64_t)cfg->max_seq;
@@ -405,6 +512,7 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
 int lckv_cache_free(lckv_cache_t* cache)
 {
     if (!cache) return LCKV_EINVAL;
+    drop_graph(cache);
     delete cache;
     return LCKV_OK;
 }
@@ -443,7 +551,7 @@ int lckv_cache_reset(lckv_cache_t* c, const int32_t* host_lens, int32_t batch, v
         for (int b = 0; b < batch; ++b) c->h_lens[b] = 0;
         if (!cuda_ok(cudaMemsetAsync(c->d_lens, 0, (size_t)batch * 4, st))) return LCKV_ECUDA;
     }
-    if (!cuda_ok(cudaMemsetAsync(c->d_counters, 0, (size_t)c->n_workers * 4, st))) return LCKV_ECUDA;
+    if (!cuda_ok(cudaMemsetAsync(c->d_counters, 0, 2 * (size_t)c->n_workers * 4, st))) return LCKV_ECUDA;
     if (!cuda_ok(cudaMemsetAsync(c->d_status, 0, 4, st))) return LCKV_ECUDA;
     return LCKV_OK;
 }
@@ -482,7 +590,10 @@ int lckv_append_kv(lckv_cache_t* c, int32_t slot, const void* k_new, const void*
     if (max_len(c, batch) + 1 > c->cfg.max_seq) return LCKV_ECAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
     if (int rc = launch_append(c, slot, k_new, v_new, batch, st)) return rc;
-    if (advance_len) return launch_advance(c, batch, st);
+    if (advance_len) {
+        if (int rc = launch_advance(c, batch, st)) return rc;
+        mirror_advance(c, batch);
+    }
     return LCKV_OK;
 }
 
@@ -510,8 +621,8 @@ int lckv_layer_stack_step(lckv_cache_t* c, const void* const* q_layers, void* co
         if (c->plan.write_slot[l] >= 0 && (!k_new_layers[l] || !v_new_layers[l])) return LCKV_EINVAL;
     }
     if (max_len(c, batch) + 1 > c->cfg.max_seq) return LCKV_ECAPACITY;
-    return enqueue_step(c, q_layers, out_layers, k_new_layers, v_new_layers, batch,
-                        static_cast<cudaStream_t>(stream));
+    return run_step(c, q_layers, out_layers, k_new_layers, v_new_layers, batch,
+                    static_cast<cudaStream_t>(stream));
 }
 
 int lckv_layer_stack_step_host(lckv_cache_t* c, const void* const* q_host, void* const* out_host,
@@ -551,7 +662,7 @@ int lckv_layer_stack_step_host(lckv_cache_t* c, const void* const* q_host, void*
             ++kv_i;
         }
     }
-    if (int rc = enqueue_step(c, dq.data(), dout.data(), dk.data(), dv.data(), batch, st)) return rc;
+    if (int rc = run_step(c, dq.data(), dout.data(), dk.data(), dv.data(), batch, st)) return rc;
     for (int l = 0; l < L; ++l)
         if (!cuda_ok(cudaMemcpyAsync(out_host[l], dout[l], o_bytes, cudaMemcpyDeviceToHost, st)))
             return LCKV_ECUDA;
@@ -681,6 +792,7 @@ extern "C" int lckv_decode_attention_static(const void* k, const void* v, const 
     p.mode = mode;
     p.n_workers = n_workers;
     p.out_f32 = out_dtype;
+    p.early_kv = 0;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
     p.scale_log2 = scale * 1.4426950408889634f;
     if (head_dim == 128)

@@ -49,6 +49,9 @@ struct AttnParams {
     int64_t T_cap;
     int32_t B, H_q, H_kv, mode, n_workers, out_f32;
     float scale_log2;         // softmax scale * log2(e)
+    int32_t early_kv;         // 1: the launcher guarantees that the plan tables and the visible K/V
+                              // rows were final before the PREVIOUS kernel in the stream started,
+                              // so the first copies may be issued before the dependency wait
 };
 
 struct TileCursor {
@@ -103,36 +106,25 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
     }
     __syncwarp();
 
-    // Rows that see nothing (diagonal-masked first token): the zero dummy KV gives o = 0, lse = 0.
-    for (int b = w; b < p.B; b += p.n_workers) {
-        if (__ldg(p.lens + b) + p.mode == 0) {
-            const int esz = p.out_f32 ? 4 : 2;
-            const int n16 = H * D * esz / 16;
-            uint4* o16 = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.out) +
-                                                  (size_t)b * H * D * esz);
-            for (int i = lane; i < n16; i += 32) o16[i] = make_uint4(0, 0, 0, 0);
-            if (p.lse)
-                for (int i = lane; i < H; i += 32) p.lse[(size_t)b * H + i] = 0.f;
-        }
-    }
+    if (!p.early_kv) pdl_wait_then_release();
 
     const uint64_t total = (uint64_t)__ldg(p.pre + p.B) * (uint64_t)H;
-    if (total == 0) return;
     const uint64_t n_eff = total < (uint64_t)p.n_workers ? total : (uint64_t)p.n_workers;
-    if ((uint64_t)w >= n_eff) return;
-    const uint64_t lo = (uint64_t)w * total / n_eff;
-    const uint64_t hi = (uint64_t)(w + 1) * total / n_eff;
-    const uint32_t n_tiles = (uint32_t)(hi - lo);
-    const uint32_t n_items = 2 * n_tiles;
-
+    const bool has_work = (uint64_t)w < n_eff;
+    uint64_t lo = 0, hi = 0;
     TileCursor cc;
-    cc.b = __ldg(p.start_b + w);
-    cursor_load(cc, p);
-    {
+    cc.b = 0; cc.h = 0; cc.t = 0; cc.nt = 0; cc.nv = 0;
+    if (has_work) {
+        lo = (uint64_t)w * total / n_eff;
+        hi = (uint64_t)(w + 1) * total / n_eff;
+        cc.b = __ldg(p.start_b + w);
+        cursor_load(cc, p);
         const uint64_t rel = lo - (uint64_t)__ldg(p.pre + cc.b) * (uint64_t)H;
         cc.h = (int32_t)(rel / cc.nt);
         cc.t = (uint32_t)(rel % cc.nt);
     }
+    const uint32_t n_tiles = (uint32_t)(hi - lo);
+    const uint32_t n_items = 2 * n_tiles;
     TileCursor ci = cc;
 
     uint32_t issued = 0, islot = 0;
@@ -154,6 +146,22 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
         const uint32_t pro = n_items < (uint32_t)NS ? n_items : (uint32_t)NS;
         while (issued < pro) issue();
     }
+    if (p.early_kv) pdl_wait_then_release();
+
+    // Rows that see nothing (diagonal-masked first token): the zero dummy KV gives o = 0, lse = 0.
+    for (int b = w; b < p.B; b += p.n_workers) {
+        if (__ldg(p.lens + b) + p.mode == 0) {
+            const int esz = p.out_f32 ? 4 : 2;
+            const int n16 = H * D * esz / 16;
+            uint4* o16 = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.out) +
+                                                  (size_t)b * H * D * esz);
+            for (int i = lane; i < n16; i += 32) o16[i] = make_uint4(0, 0, 0, 0);
+            if (p.lse)
+                for (int i = lane; i < H; i += 32) p.lse[(size_t)b * H + i] = 0.f;
+        }
+    }
+
+    if (!has_work) return;
 
     const int grp = lane / LPR;  // which of the RPI rows of a load this lane reads
     const int a = lane % LPR;    // which 16 bytes of the row

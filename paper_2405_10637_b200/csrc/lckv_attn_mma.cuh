@@ -150,38 +150,26 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
     }
     __syncwarp();
 
-    // Sequences that see nothing: zero rows (zero dummy KV), lse 0.
-    for (int b = w; b < p.B; b += p.n_workers) {
-        if (__ldg(p.lens + b) + p.mode == 0) {
-            const int esz = p.out_f32 ? 4 : 2;
-            const int n16 = mp.n_q_heads * D * esz / 16;
-            uint4* o16 = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.out) +
-                                                  (size_t)b * mp.n_q_heads * D * esz);
-            for (int i = lane; i < n16; i += 32) o16[i] = make_uint4(0, 0, 0, 0);
-            if (p.lse)
-                for (int i = lane; i < mp.n_q_heads; i += 32)
-                    p.lse[(size_t)b * mp.n_q_heads + i] = 0.f;
-        }
-    }
+    if (!p.early_kv) pdl_wait_then_release();
 
     const uint64_t total = (uint64_t)__ldg(p.pre + p.B) * (uint64_t)H;
-    if (total == 0) return;
     const uint64_t n_eff = total < (uint64_t)p.n_workers ? total : (uint64_t)p.n_workers;
-    if ((uint64_t)w >= n_eff) return;
-    const uint64_t lo = (uint64_t)w * total / n_eff;
-    const uint64_t hi = (uint64_t)(w + 1) * total / n_eff;
-    const uint32_t n_tiles = (uint32_t)(hi - lo);
-    const uint32_t n_items = 2 * n_tiles;
-
+    const bool has_work = (uint64_t)w < n_eff;
+    uint64_t lo = 0, hi = 0;
     RowCursor cc;
-    cc.b = __ldg(p.start_b + w);
-    rcursor_load(cc, p);
-    {
+    cc.b = 0; cc.h = 0; cc.t = 0; cc.nt = 0; cc.nv = 0; cc.kvh = 0; cc.sub = 0; cc.row = 0;
+    if (has_work) {
+        lo = (uint64_t)w * total / n_eff;
+        hi = (uint64_t)(w + 1) * total / n_eff;
+        cc.b = __ldg(p.start_b + w);
+        rcursor_load(cc, p);
         const uint64_t rel = lo - (uint64_t)__ldg(p.pre + cc.b) * (uint64_t)H;
         cc.h = (int32_t)(rel / cc.nt);
         cc.t = (uint32_t)(rel % cc.nt);
+        rcursor_seek(cc, p, mp.groups_per_kv, R);
     }
-    rcursor_seek(cc, p, mp.groups_per_kv, R);
+    const uint32_t n_tiles = (uint32_t)(hi - lo);
+    const uint32_t n_items = 2 * n_tiles;
     RowCursor ci = cc;
 
     uint32_t issued = 0, islot = 0;
@@ -203,6 +191,23 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
         const uint32_t pro = n_items < (uint32_t)NS ? n_items : (uint32_t)NS;
         while (issued < pro) issue();
     }
+    if (p.early_kv) pdl_wait_then_release();
+
+    // Sequences that see nothing: zero rows (zero dummy KV), lse 0.
+    for (int b = w; b < p.B; b += p.n_workers) {
+        if (__ldg(p.lens + b) + p.mode == 0) {
+            const int esz = p.out_f32 ? 4 : 2;
+            const int n16 = mp.n_q_heads * D * esz / 16;
+            uint4* o16 = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.out) +
+                                                  (size_t)b * mp.n_q_heads * D * esz);
+            for (int i = lane; i < n16; i += 32) o16[i] = make_uint4(0, 0, 0, 0);
+            if (p.lse)
+                for (int i = lane; i < mp.n_q_heads; i += 32)
+                    p.lse[(size_t)b * mp.n_q_heads + i] = 0.f;
+        }
+    }
+
+    if (!has_work) return;
 
     uint32_t cslot = 0, cphase = 0;
     bool ok = true;

@@ -94,6 +94,15 @@ __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const void* tmap,
         : "memory");
 }
 
+// Programmatic dependent launch: wait until every kernel this launch depends on has completed and
+// its writes are visible, then allow the next kernel in the stream to start being scheduled.
+// Both are no-ops for a kernel launched without the programmatic-serialization attribute.
+__device__ __forceinline__ void pdl_wait_then_release()
+{
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+
 __device__ __forceinline__ float ex2(float x)
 {
     float y;

@@ -218,3 +218,39 @@ def test_alu_kernel_forced_for_grouped_heads():
     assert c.cache.info.kernel_kind == 1
     c.step()
     c.close()
+
+
+@pytest.mark.parametrize("shape", ["mha", "gqa"])
+def test_graph_replay_steps_match(shape):
+    """use_graph = 1: the step is captured once and replayed while the argument pointers repeat;
+    lengths live on the device, so every replay sees the grown caches."""
+    kw = dict(Hq=8, Hkv=8, d=128, std=1.0) if shape == "mha" else dict(Hq=16, Hkv=2, d=64, std=0.25)
+    torch.cuda.set_stream(torch.cuda.Stream())   # the legacy default stream cannot be captured
+    c = Case(L=5, w=2, lens=[0, 3, 16, 200, 333], T_cap=400, seed=77, use_graph=1, **kw)
+    dev = c.cache.device
+    odt = torch.bfloat16
+    # fixed device buffers, new contents each step -> same pointers -> replay
+    q = [torch.empty((c.B, c.Hq, c.d), dtype=torch.bfloat16, device=dev) for _ in range(c.L)]
+    kn = [torch.empty((c.B, c.Hkv, c.d), dtype=torch.bfloat16, device=dev)
+          if c.plan["write_slot"][l] >= 0 else None for l in range(c.L)]
+    vn = [None if t is None else torch.empty_like(t) for t in kn]
+    outs = [torch.empty((c.B, c.Hq, c.d), dtype=odt, device=dev) for _ in range(c.L)]
+    for step in range(4):
+        hq, hk, hv = c.step_inputs()
+        for l in range(c.L):
+            q[l].copy_(hq[l])
+            if kn[l] is not None:
+                kn[l].copy_(hk[l]); vn[l].copy_(hv[l])
+        c.cache.lckv_layer_stack_step(q, outs, kn, vn)
+        torch.cuda.synchronize()
+        want, _ = orc.stack_step(c.L, c.w, [syn.bits(t) for t in hq],
+                                 [None if t is None else syn.bits(t) for t in hk],
+                                 [None if t is None else syn.bits(t) for t in hv],
+                                 c.hK, c.hV, c.lens, c.scale)
+        c.step_no += 1
+        for l in range(c.L):
+            compare(outs[l], want[l], f"graph step {step} layer {l}")
+        c.check_state()
+    c.close()
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(torch.cuda.default_stream())
