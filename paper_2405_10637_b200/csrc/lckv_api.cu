@@ -3,6 +3,7 @@
 
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <vector>
@@ -88,6 +89,7 @@ struct lckv_cache {
     std::vector<int32_t> h_lens;  // host mirror of the device lengths
     int n_kv_layers;
     std::vector<CUtensorMap> tm_k, tm_v;  // per slot, tensor-core kernel only
+    double l2_keep_bytes;                 // how much of a re-read slot to hold in L2 (0 = off)
     int ws_parity;                        // which half of the split-K workspace the next launch uses
     size_t partials_half_floats;          // floats in one half of the partial records
     // CUDA graph of one step, valid for the argument pointers it was captured with
@@ -247,7 +249,7 @@ cudaError_t launch_pdl(void (*kernel)(KArgs...), int grid, int block, size_t sme
 // early: the previous kernel in the stream is an attention launch of the same step and this one
 // reads only rows that were final before it (condensed mode), so its first copies need not wait.
 int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out, float* lse,
-                     int batch, cudaStream_t st, bool early = false)
+                     int batch, cudaStream_t st, bool early = false, float l2_keep = 0.f)
 {
     lckv::AttnParams p;
     p.K = slot_k(c, slot);
@@ -272,6 +274,7 @@ int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out
     p.out_f32 = c->cfg.out_dtype;
     p.scale_log2 = c->scale_log2;
     p.early_kv = early ? 1 : 0;
+    p.l2_keep = l2_keep;
     cudaError_t e;
     if (c->kernel_kind == 2) {
         lckv::MmaParams mp;
@@ -319,6 +322,18 @@ void mirror_advance(lckv_cache* c, int batch)
     for (int b = 0; b < batch; ++b) c->h_lens[b] += 1;
 }
 
+// Fraction of a re-read slot's lines to mark evict-last, judged from the host mirror of the
+// lengths, in sixteenths (so that a captured step stays valid while the caches grow a little).
+float step_keep_frac(const lckv_cache* c, int batch)
+{
+    int64_t rows = 0;
+    for (int b = 0; b < batch; ++b) rows += c->h_lens[b];
+    const double bytes = (double)rows * 4.0 * c->cfg.n_kv_heads * c->cfg.head_dim;
+    if (bytes <= 0 || c->l2_keep_bytes <= 0) return 0.f;
+    const double f = std::fmin(1.0, c->l2_keep_bytes / bytes);
+    return (float)(std::floor(f * 16.0) / 16.0);
+}
+
 // The launches of one step, in the order the header states.
 int enqueue_step(lckv_cache* c, const void* const* q, void* const* out, const void* const* kn,
                  const void* const* vn, int batch, cudaStream_t st)
@@ -329,6 +344,11 @@ int enqueue_step(lckv_cache* c, const void* const* q, void* const* out, const vo
     // workspace half 0; this also makes a captured step replayable.
     c->ws_parity = 0;
     if (int rc = launch_plan(c, batch, st)) return rc;
+    // A slot that several layers read in this step is worth keeping in L2 between their passes, as
+    // far as it fits: mark that fraction of its lines evict-last.  A slot read once is streamed.
+    const float keep_frac = step_keep_frac(c, batch);
+    std::vector<int> readers(pl.n_slots, 0);
+    for (int l = 0; l < L; ++l) readers[pl.read_slot[l]] += 1;
     bool prev_attn = false;
     for (int l = 0; l < L; ++l) {
         if (pl.write_slot[l] >= 0 && pl.write_before[l]) {
@@ -336,8 +356,9 @@ int enqueue_step(lckv_cache* c, const void* const* q, void* const* out, const vo
             prev_attn = false;
         }
         const bool early = prev_attn && pl.mode[l] == LCKV_MODE_CONDENSED;
+        const float keep = readers[pl.read_slot[l]] > 1 ? keep_frac : 0.f;
         if (int rc = launch_attention(c, pl.read_slot[l], pl.mode[l], q[l], out[l], nullptr, batch,
-                                      st, early))
+                                      st, early, keep))
             return rc;
         prev_attn = true;
     }
@@ -361,8 +382,9 @@ int step_with_graph(lckv_cache* c, const void* const* q, void* const* out, const
 {
     const int L = c->cfg.n_layers;
     std::vector<const void*> key;
-    key.reserve(4 * L + 1);
+    key.reserve(4 * L + 2);
     key.push_back(reinterpret_cast<const void*>((uintptr_t)batch));
+    key.push_back(reinterpret_cast<const void*>((uintptr_t)(step_keep_frac(c, batch) * 16.f)));
     for (int l = 0; l < L; ++l) {
         key.push_back(q[l]);
         key.push_back(out[l]);
@@ -476,6 +498,15 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     c->d_status = reinterpret_cast<int32_t*>(c->base + c->lay.off_status);
     c->d_partials = reinterpret_cast<float*>(c->base + c->lay.off_partials);
     c->h_lens.assign(cfg->max_batch, 0);
+    {
+        // About half of the L2 (measured optimum on B200, 126 MB L2: 60-70 MB; more than that and
+        // the evict-last lines start displacing each other).  LCKV_L2_KEEP_MB overrides (0 = off).
+        int dev = 0, l2 = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&l2, cudaDevAttrL2CacheSize, dev);
+        const char* env = getenv("LCKV_L2_KEEP_MB");
+        c->l2_keep_bytes = env ? atof(env) * 1e6 : 0.52 * (double)l2;
+    }
     c->ws_parity = 0;
     c->partials_half_floats = 2 * (size_t)c->n_workers * partial_record_floats(*cfg);
     c->graph_exec = nullptr;
@@ -793,6 +824,7 @@ extern "C" int lckv_decode_attention_static(const void* k, const void* v, const 
     p.n_workers = n_workers;
     p.out_f32 = out_dtype;
     p.early_kv = 0;
+    p.l2_keep = 0.f;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
     p.scale_log2 = scale * 1.4426950408889634f;
     if (head_dim == 128)

@@ -49,6 +49,8 @@ struct AttnParams {
     int64_t T_cap;
     int32_t B, H_q, H_kv, mode, n_workers, out_f32;
     float scale_log2;         // softmax scale * log2(e)
+    float l2_keep;            // fraction of the cache lines to keep in L2 for the next layer's
+                              // pass over the same cache (0: stream everything)
     int32_t early_kv;         // 1: the launcher guarantees that the plan tables and the visible K/V
                               // rows were final before the PREVIOUS kernel in the stream started,
                               // so the first copies may be issued before the dependency wait
@@ -127,6 +129,7 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
     const uint32_t n_items = 2 * n_tiles;
     TileCursor ci = cc;
 
+    const uint64_t l2pol = make_l2_policy(p.l2_keep);
     uint32_t issued = 0, islot = 0;
     auto issue = [&]() {
         const int rows = min(R, ci.nv - (int)ci.t * R);
@@ -136,7 +139,7 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
             base + (((int64_t)ci.b * p.H_kv + ci.h / g) * p.T_cap + (int64_t)ci.t * R) * D;
         if (lane == 0) {
             mbar_expect_tx(bars + 8 * islot, bytes);
-            bulk_g2s(ring + islot * kAluSlotBytes, src, bytes, bars + 8 * islot);
+            bulk_g2s_hint(ring + islot * kAluSlotBytes, src, bytes, bars + 8 * islot, l2pol);
         }
         if (issued & 1) cursor_next(ci, p, H);
         ++issued;

@@ -172,6 +172,7 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
     const uint32_t n_items = 2 * n_tiles;
     RowCursor ci = cc;
 
+    const uint64_t l2pol = make_l2_policy(p.l2_keep);
     uint32_t issued = 0, islot = 0;
     auto issue = [&]() {
         const int64_t row = ci.row;
@@ -180,8 +181,8 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
             mbar_expect_tx(bars + 8 * islot, kMmaSlotBytes);
 #pragma unroll
             for (int bx = 0; bx < NBOX; ++bx)
-                tma_load_2d(ring + islot * kMmaSlotBytes + bx * BOX_BYTES, tm, bx * 64, (int32_t)row,
-                            bars + 8 * islot);
+                tma_load_2d_hint(ring + islot * kMmaSlotBytes + bx * BOX_BYTES, tm, bx * 64,
+                                 (int32_t)row, bars + 8 * islot, l2pol);
         }
         if (issued & 1) rcursor_next(ci, p, H, mp.groups_per_kv, R);
         ++issued;

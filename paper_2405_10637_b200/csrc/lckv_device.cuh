@@ -83,6 +83,43 @@ __device__ __forceinline__ void bulk_g2s(uint32_t dst_smem, const void* src, uin
         : "memory");
 }
 
+// L2 eviction policy for the cache rows: a fixed (address-hashed) fraction `keep` of the lines is
+// marked evict-last so that it survives until the next layer re-reads the same cache, the rest is
+// marked evict-first (pure streaming).  keep <= 0 gives all evict-first.
+__device__ __forceinline__ uint64_t make_l2_policy(float keep)
+{
+    uint64_t pol;
+    if (keep > 0.f) {
+        keep = fminf(keep, 1.0f);
+        asm volatile("createpolicy.fractional.L2::evict_last.L2::evict_first.b64 %0, %1;"
+                     : "=l"(pol)
+                     : "f"(keep));
+    } else {
+        asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+    }
+    return pol;
+}
+
+__device__ __forceinline__ void bulk_g2s_hint(uint32_t dst_smem, const void* src, uint32_t bytes,
+                                              uint32_t bar, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint "
+        "[%0], [%1], %2, [%3], %4;"
+        ::"r"(dst_smem), "l"(src), "r"(bytes), "r"(bar), "l"(policy)
+        : "memory");
+}
+
+__device__ __forceinline__ void tma_load_2d_hint(uint32_t dst_smem, const void* tmap, int32_t x,
+                                                 int32_t y, uint32_t bar, uint64_t policy)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.tile.mbarrier::complete_tx::bytes"
+        ".L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+        ::"r"(dst_smem), "l"(tmap), "r"(x), "r"(y), "r"(bar), "l"(policy)
+        : "memory");
+}
+
 // 2-D tiled TMA load (tensor map), coordinates {x = element column, y = row}.  No multicast.
 __device__ __forceinline__ void tma_load_2d(uint32_t dst_smem, const void* tmap, int32_t x,
                                             int32_t y, uint32_t bar)
