@@ -67,19 +67,27 @@ def workload_params(args):
     if args.context:
         p["lo"] = p["hi"] = args.context
         p["t_cap"] = args.context
-    # room for the tokens the run itself appends (lengths grow by one per step)
-    p["t_cap"] += max(64, args.steps + args.warmup + 8)
+    if args.stream_sink:
+        # sink + recent-window caches of exactly t_cap rows, already full: every sequence is three
+        # cache sizes long, so appends wrap around the ring and reads cover the whole cache
+        p["lo"] = p["hi"] = 3 * p["t_cap"]
+    else:
+        # room for the tokens the run itself appends (lengths grow by one per step)
+        p["t_cap"] += max(64, args.steps + args.warmup + 8)
     return wl, p
 
 
-def step_kv_bytes(wl, plan_modes, lens, batch, grown=0):
+def step_kv_bytes(wl, plan_modes, lens, batch, grown=0, cap=0):
     """Algorithmic K+V bytes one step reads: every layer reads its visible rows once.
     `grown` = tokens appended to every sequence since `lens` was set."""
     per_row = 4 * wl.n_kv_heads * wl.head_dim
-    s = int(np.asarray(lens[:batch], np.int64).sum()) + grown * batch
+    ln = np.asarray(lens[:batch], np.int64) + grown
     total = 0
     for m in plan_modes:
-        total += per_row * (s + m * batch)
+        vis = ln + m
+        if cap:
+            vis = np.minimum(vis, cap)
+        total += per_row * int(vis.sum())
     return total
 
 
@@ -239,7 +247,8 @@ def run_ours(args):
     L = wl.n_layers
     cfg = lk.make_config(L, wl.n_warmup, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, B, T_cap,
                          host_staging=1, use_graph=1 if args.graph else 0,
-                         top_variant=args.top_variant)
+                         top_variant=args.top_variant, stream_sink=args.stream_sink)
+    cap = T_cap if args.stream_sink else 0
     cache = lk.Cache(cfg, device=dev)
     plan = lk.lckv_plan(L, wl.n_warmup, args.top_variant)
     info = cache.info
@@ -276,7 +285,7 @@ def run_ours(args):
             f()
         barrier()
         ms = time_steps(f, k, stream) / k
-        by = sum(step_kv_bytes(wl, modes, lens, b, warm + i) for i in range(k)) / k
+        by = sum(step_kv_bytes(wl, modes, lens, b, warm + i, cap) for i in range(k)) / k
         return ms, by
 
     def barrier():
@@ -313,7 +322,7 @@ def run_ours(args):
     torch.cuda.synchronize()
     ms_attn = time_steps(attn, n_launch, stream) / n_launch
     io_bytes = 2 * B * wl.n_q_heads * wl.head_dim * 2
-    alg_bytes = 4 * wl.n_kv_heads * wl.head_dim * int(lens.astype(np.int64).sum()) + io_bytes
+    alg_bytes = step_kv_bytes(wl, [0], lens, B, 0, cap) + io_bytes
     peak, peak_kind = measured_peaks()
     achieved = alg_bytes / (ms_attn * 1e-3) / 1e9
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
@@ -353,7 +362,7 @@ def run_ours(args):
 
     # ---- CPU baseline: the checker on a bounded sample (rank 0, N = 1 only) --------------------
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.stream_sink:
         rows = min(args.ref_rows, B)
         Ks = [syn.bits(cache.slot_tensors(s)[0][:rows]) for s in range(info.n_slots)]
         Vs = [syn.bits(cache.slot_tensors(s)[1][:rows]) for s in range(info.n_slots)]
@@ -372,7 +381,8 @@ def run_ours(args):
             "config": {"workload": workload_name(wl, p), "l2": "inputs larger than L2"
                        if 2 * info.slot_bytes > 2 * 126e6 else "L2-resident cache: warm",
                        "kv_bytes_per_step": bytes_step, "footprint_slots": info.n_slots,
-                       "top_variant": args.top_variant, "graph": bool(args.graph)},
+                       "top_variant": args.top_variant, "graph": bool(args.graph),
+                       "stream_sink": args.stream_sink},
             "frac_of_8TBs": value / world / NOMINAL_HBM_GBS,
             "clocks": clocks, "e2e": e2e, "gpu_launches": info.launches_per_step * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "sweep": sweep,
@@ -395,6 +405,8 @@ def main():
     ap.add_argument("--warmup-layers", type=int, default=None, help="override w")
     ap.add_argument("--top-variant", type=int, default=0)
     ap.add_argument("--graph", type=int, default=1)
+    ap.add_argument("--stream-sink", type=int, default=0,
+                    help="s > 0: sink + recent-window caches with s sink tokens, cache size = context")
     ap.add_argument("--ref-rows", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()

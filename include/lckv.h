@@ -71,6 +71,11 @@ typedef struct {
     int32_t use_graph;     /* 1: lckv_layer_stack_step replays a CUDA graph when the argument
                               pointers repeat from the previous call (needs a stream other
                               than the legacy default stream; otherwise plain launches)      */
+    int32_t stream_sink;   /* 0 = off.  s >= 1: StreamingLLM-style caches (paper Section 3.3): every
+                              slot keeps the first s tokens ("attention sinks") and the most
+                              recent max_seq - s tokens; token t >= max_seq overwrites row
+                              s + (t - s) mod (max_seq - s).  Lengths keep counting all tokens;
+                              LCKV_ECAPACITY is never returned.  Needs 1 <= s < max_seq.     */
     int32_t kernel_kind;   /* 0 = choose (tensor-core kernel when the query group is a dense
                               MMA tile, else the FP32-ALU kernel); 1 = force FP32-ALU        */
 } lckv_config_t;

@@ -21,6 +21,10 @@
  *   top_variant 0  the shared cache is the cache of layer L-1 itself, even
  *                  when that layer is a warmup layer (Section 2.1, literal);
  *   top_variant 1  the shared cache is fed by the topmost non-warmup layer;
+ *   n_sink         0: caches grow without bound (up to T_cap rows).  s >= 1: the cache keeps the
+ *                  first s tokens and the most recent T_cap - s tokens (the StreamingLLM policy
+ *                  the paper combines with its model in Section 3.3); the evicted token's row is
+ *                  reused, row(t) = t for t < T_cap, else s + (t - s) mod (T_cap - s).
  *   always_sink    0: the zero dummy key/value is used only when a query sees
  *                  nothing (first token, Section 2.1); 1: it is a permanent
  *                  extra column of every row (alternative reading, CPU only).
@@ -165,15 +169,17 @@ int lckv_oracle_attend_row(const uint16_t* q, const uint16_t* K, const uint16_t*
  */
 int lckv_oracle_decode_attention(const uint16_t* q, const uint16_t* K, const uint16_t* V,
                                  const int32_t* lens, int B, int H_q, int H_kv, int64_t T_cap,
-                                 int d, int mode, double scale, int always_sink, double* out,
-                                 double* lse)
+                                 int d, int mode, double scale, int always_sink, int n_sink,
+                                 double* out, double* lse)
 {
     if (B < 0 || H_q < 1 || H_kv < 1 || H_q % H_kv != 0 || d < 1) return LCKV_ORACLE_EINVAL;
     if (mode != 0 && mode != 1) return LCKV_ORACLE_EINVAL;
     int g = H_q / H_kv;
     for (int b = 0; b < B; ++b) {
-        if (lens[b] < 0 || (int64_t)lens[b] + mode > T_cap) return LCKV_ORACLE_ECAPACITY;
+        if (lens[b] < 0) return LCKV_ORACLE_ECAPACITY;
+        if (n_sink <= 0 && (int64_t)lens[b] + mode > T_cap) return LCKV_ORACLE_ECAPACITY;
     }
+    if (n_sink < 0 || (n_sink > 0 && n_sink >= T_cap)) return LCKV_ORACLE_EINVAL;
     int64_t rows = (int64_t)B * H_q;
 #pragma omp parallel
     {
@@ -182,7 +188,10 @@ int lckv_oracle_decode_attention(const uint16_t* q, const uint16_t* K, const uin
         for (int64_t r = 0; r < rows; ++r) {
             int b = (int)(r / H_q), h = (int)(r % H_q);
             int kvh = h / g;
+            /* Section 3.3: with the sink + recent-window policy the cache holds at most T_cap
+             * tokens; all of them precede the query (or are the query's own, standard mode). */
             int64_t n_vis = (int64_t)lens[b] + mode;
+            if (n_sink > 0 && n_vis > T_cap) n_vis = T_cap;
             const uint16_t* Kp = K + (((int64_t)b * H_kv + kvh) * T_cap) * d;
             const uint16_t* Vp = V + (((int64_t)b * H_kv + kvh) * T_cap) * d;
             attend_row(q + r * d, Kp, Vp, n_vis, d, scale, always_sink, out + r * d,
@@ -199,13 +208,18 @@ int lckv_oracle_decode_attention(const uint16_t* q, const uint16_t* K, const uin
  * token so they are not recomputed).  Lengths are not changed here.
  */
 int lckv_oracle_append(uint16_t* K, uint16_t* V, const uint16_t* k_new, const uint16_t* v_new,
-                       const int32_t* lens, int B, int H_kv, int64_t T_cap, int d)
+                       const int32_t* lens, int B, int H_kv, int64_t T_cap, int d, int n_sink)
 {
+    if (n_sink < 0 || (n_sink > 0 && n_sink >= T_cap)) return LCKV_ORACLE_EINVAL;
     for (int b = 0; b < B; ++b)
-        if (lens[b] < 0 || (int64_t)lens[b] >= T_cap) return LCKV_ORACLE_ECAPACITY;
+        if (lens[b] < 0 || (n_sink <= 0 && (int64_t)lens[b] >= T_cap)) return LCKV_ORACLE_ECAPACITY;
     for (int b = 0; b < B; ++b)
         for (int h = 0; h < H_kv; ++h) {
-            int64_t dst = ((((int64_t)b * H_kv + h) * T_cap) + lens[b]) * d;
+            /* token t goes to row t; once the cache is full (streaming policy) it replaces the
+             * oldest token that is not one of the first n_sink */
+            int64_t row = lens[b];
+            if (n_sink > 0 && row >= T_cap) row = n_sink + (row - n_sink) % (T_cap - n_sink);
+            int64_t dst = ((((int64_t)b * H_kv + h) * T_cap) + row) * d;
             int64_t src = ((int64_t)b * H_kv + h) * d;
             memcpy(K + dst, k_new + src, sizeof(uint16_t) * (size_t)d);
             memcpy(V + dst, v_new + src, sizeof(uint16_t) * (size_t)d);
@@ -234,7 +248,7 @@ int lckv_oracle_stack_step(int L, int w, int top_variant, const uint16_t* const*
                            const uint16_t* const* k_new_layers,
                            const uint16_t* const* v_new_layers, uint16_t* const* K_slots,
                            uint16_t* const* V_slots, int32_t* lens, int B, int H_q, int H_kv,
-                           int64_t T_cap, int d, double scale, int always_sink,
+                           int64_t T_cap, int d, double scale, int always_sink, int n_sink,
                            double* const* out_layers, double* const* lse_layers)
 {
     int32_t* plan = (int32_t*)malloc(sizeof(int32_t) * 5 * (size_t)L);
@@ -245,23 +259,23 @@ int lckv_oracle_stack_step(int L, int w, int top_variant, const uint16_t* const*
     int rc = lckv_oracle_plan(L, w, top_variant, is_w, rs, md, ws, wb, &n_slots);
     if (rc) { free(plan); return rc; }
     for (int b = 0; b < B; ++b)
-        if (lens[b] < 0 || (int64_t)lens[b] + 1 > T_cap) { free(plan); return LCKV_ORACLE_ECAPACITY; }
+        if (lens[b] < 0 || (n_sink <= 0 && (int64_t)lens[b] + 1 > T_cap)) { free(plan); return LCKV_ORACLE_ECAPACITY; }
     for (int l = 0; l < L; ++l)
         if (ws[l] >= 0 && (!k_new_layers[l] || !v_new_layers[l])) { free(plan); return LCKV_ORACLE_EINVAL; }
 
     for (int l = 0; l < L && rc == 0; ++l) {
         if (ws[l] >= 0 && wb[l])
             rc = lckv_oracle_append(K_slots[ws[l]], V_slots[ws[l]], k_new_layers[l],
-                                    v_new_layers[l], lens, B, H_kv, T_cap, d);
+                                    v_new_layers[l], lens, B, H_kv, T_cap, d, n_sink);
         if (rc) break;
         rc = lckv_oracle_decode_attention(q_layers[l], K_slots[rs[l]], V_slots[rs[l]], lens, B,
-                                          H_q, H_kv, T_cap, d, md[l], scale, always_sink,
+                                          H_q, H_kv, T_cap, d, md[l], scale, always_sink, n_sink,
                                           out_layers[l], lse_layers ? lse_layers[l] : NULL);
     }
     for (int l = 0; l < L && rc == 0; ++l)
         if (ws[l] >= 0 && !wb[l])
             rc = lckv_oracle_append(K_slots[ws[l]], V_slots[ws[l]], k_new_layers[l],
-                                    v_new_layers[l], lens, B, H_kv, T_cap, d);
+                                    v_new_layers[l], lens, B, H_kv, T_cap, d, n_sink);
     if (rc == 0)
         for (int b = 0; b < B; ++b) lens[b] += 1;
     free(plan);

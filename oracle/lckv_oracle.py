@@ -29,15 +29,15 @@ def lib():
         L.lckv_oracle_attend_row.restype = C.c_int
         L.lckv_oracle_decode_attention.argtypes = [u16p, u16p, u16p, i32p, C.c_int, C.c_int,
                                                    C.c_int, C.c_int64, C.c_int, C.c_int,
-                                                   C.c_double, C.c_int, f64p, f64p]
+                                                   C.c_double, C.c_int, C.c_int, f64p, f64p]
         L.lckv_oracle_decode_attention.restype = C.c_int
         L.lckv_oracle_append.argtypes = [u16p, u16p, u16p, u16p, i32p, C.c_int, C.c_int,
-                                         C.c_int64, C.c_int]
+                                         C.c_int64, C.c_int, C.c_int]
         L.lckv_oracle_append.restype = C.c_int
         pp = C.POINTER(C.c_void_p)
         L.lckv_oracle_stack_step.argtypes = [C.c_int, C.c_int, C.c_int, pp, pp, pp, pp, pp, i32p,
                                              C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int,
-                                             C.c_double, C.c_int, pp, pp]
+                                             C.c_double, C.c_int, C.c_int, pp, pp]
         L.lckv_oracle_stack_step.restype = C.c_int
         L.lckv_oracle_num_threads.restype = C.c_int
         _LIB = L
@@ -95,7 +95,7 @@ def attend_row(q, K, V, scale, always_sink=False, want_probs=False):
     return (o, float(lse[0]), probs) if want_probs else (o, float(lse[0]))
 
 
-def decode_attention(q, K, V, lens, mode, scale, always_sink=False):
+def decode_attention(q, K, V, lens, mode, scale, always_sink=False, n_sink=0):
     """q [B,Hq,d], K,V [B,Hkv,Tcap,d] uint16, lens [B] int32 -> (out [B,Hq,d], lse [B,Hq]) float64."""
     q, K, V = _u16(q), _u16(K), _u16(V)
     lens = np.ascontiguousarray(lens, np.int32)
@@ -107,12 +107,12 @@ def decode_attention(q, K, V, lens, mode, scale, always_sink=False):
     rc = lib().lckv_oracle_decode_attention(_p(q, C.c_uint16), _p(K, C.c_uint16),
                                             _p(V, C.c_uint16), _p(lens, C.c_int32), B, Hq, Hkv,
                                             Tcap, d, int(mode), float(scale), int(always_sink),
-                                            _p(out, C.c_double), _p(lse, C.c_double))
+                                            int(n_sink), _p(out, C.c_double), _p(lse, C.c_double))
     _chk(rc, "decode_attention")
     return out, lse
 
 
-def append(K, V, k_new, v_new, lens):
+def append(K, V, k_new, v_new, lens, n_sink=0):
     """In place: row lens[b] of K,V [B,Hkv,Tcap,d] <- k_new, v_new [B,Hkv,d]."""
     assert K.flags.c_contiguous and V.flags.c_contiguous and K.dtype == np.uint16
     k_new, v_new = _u16(k_new), _u16(v_new)
@@ -120,7 +120,7 @@ def append(K, V, k_new, v_new, lens):
     B, Hkv, d = k_new.shape
     rc = lib().lckv_oracle_append(_p(K, C.c_uint16), _p(V, C.c_uint16), _p(k_new, C.c_uint16),
                                   _p(v_new, C.c_uint16), _p(lens, C.c_int32), B, Hkv,
-                                  K.shape[2], d)
+                                  K.shape[2], d, int(n_sink))
     _chk(rc, "append")
 
 
@@ -132,7 +132,7 @@ def _ptr_array(arrs):
 
 
 def stack_step(L, w, q_layers, k_new_layers, v_new_layers, K_slots, V_slots, lens, scale,
-               top_variant=0, always_sink=False):
+               top_variant=0, always_sink=False, n_sink=0):
     """One decode step of the whole stack; caches and lens are updated in place.
 
     q_layers: list of L arrays [B,Hq,d]; k_new_layers/v_new_layers: list of L arrays
@@ -153,6 +153,7 @@ def stack_step(L, w, q_layers, k_new_layers, v_new_layers, K_slots, V_slots, len
                                       _ptr_array(k_new_layers), _ptr_array(v_new_layers),
                                       _ptr_array(K_slots), _ptr_array(V_slots),
                                       _p(lens, C.c_int32), B, Hq, Hkv, Tcap, d, float(scale),
-                                      int(always_sink), _ptr_array(outs), _ptr_array(lses))
+                                      int(always_sink), int(n_sink), _ptr_array(outs),
+                                      _ptr_array(lses))
     _chk(rc, "stack_step")
     return outs, lses

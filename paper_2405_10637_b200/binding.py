@@ -20,7 +20,7 @@ class Config(C.Structure):
                 ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("max_batch", C.c_int32), ("max_seq", C.c_int32), ("softmax_scale", C.c_float),
                 ("top_variant", C.c_int32), ("out_dtype", C.c_int32), ("host_staging", C.c_int32),
-                ("use_graph", C.c_int32), ("kernel_kind", C.c_int32)]
+                ("use_graph", C.c_int32), ("stream_sink", C.c_int32), ("kernel_kind", C.c_int32)]
 
 
 class Info(C.Structure):
@@ -113,10 +113,10 @@ def lckv_plan(n_layers, n_warmup, top_variant=0):
 
 def make_config(n_layers, n_warmup, n_q_heads, n_kv_heads, head_dim, max_batch, max_seq,
                 softmax_scale=0.0, top_variant=0, out_dtype=0, host_staging=0, use_graph=0,
-                kernel_kind=0):
+                kernel_kind=0, stream_sink=0):
     return Config(C.sizeof(Config), n_layers, n_warmup, n_q_heads, n_kv_heads, head_dim,
                   max_batch, max_seq, softmax_scale, top_variant, out_dtype, host_staging,
-                  use_graph, kernel_kind)
+                  use_graph, stream_sink, kernel_kind)
 
 
 def lckv_cache_bytes(cfg):

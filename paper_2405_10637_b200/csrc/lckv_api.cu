@@ -109,6 +109,7 @@ int validate_config(const lckv_config_t* c)
     if (!(c->softmax_scale >= 0.f) || !std::isfinite(c->softmax_scale)) return LCKV_EINVAL;
     if (c->out_dtype != 0 && c->out_dtype != 1) return LCKV_EINVAL;
     if (c->kernel_kind != 0 && c->kernel_kind != 1) return LCKV_EINVAL;
+    if (c->stream_sink < 0 || (c->stream_sink > 0 && c->stream_sink >= c->max_seq)) return LCKV_EINVAL;
     Plan pl;
     if (int rc = make_plan(c->n_layers, c->n_warmup, c->top_variant, pl)) return rc;
     // tile counts are kept in 32 bits
@@ -213,8 +214,10 @@ uint16_t* slot_v(const lckv_cache* c, int s)
                                        (size_t)(2 * s + 1) * c->lay.slot_bytes);
 }
 
+// Longest sequence, for capacity checks; 0 in streaming mode (a ring never overflows).
 int max_len(const lckv_cache* c, int batch)
 {
+    if (c->cfg.stream_sink > 0) return 0;
     int m = 0;
     for (int b = 0; b < batch; ++b) m = c->h_lens[b] > m ? c->h_lens[b] : m;
     return m;
@@ -223,7 +226,8 @@ int max_len(const lckv_cache* c, int batch)
 int launch_plan(lckv_cache* c, int batch, cudaStream_t st)
 {
     lckv::plan_kernel<<<1, 1024, 0, st>>>(c->d_lens, batch, c->rows_per_tile, c->h_pairs,
-                                          c->n_workers, c->d_pre, c->lay.pre_stride, c->d_start);
+                                          c->n_workers, c->d_pre, c->lay.pre_stride, c->d_start,
+                                          c->cfg.max_seq);
     return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
 }
 
@@ -307,7 +311,7 @@ int launch_append(lckv_cache* c, int slot, const void* k_new, const void* v_new,
     lckv::append_kernel<<<blocks, threads, 0, st>>>(
         slot_k(c, slot), slot_v(c, slot), static_cast<const uint16_t*>(k_new),
         static_cast<const uint16_t*>(v_new), c->d_lens, batch, c->cfg.n_kv_heads, c->cfg.max_seq,
-        c->cfg.head_dim);
+        c->cfg.head_dim, c->cfg.stream_sink);
     return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
 }
 
@@ -327,7 +331,8 @@ void mirror_advance(lckv_cache* c, int batch)
 float step_keep_frac(const lckv_cache* c, int batch)
 {
     int64_t rows = 0;
-    for (int b = 0; b < batch; ++b) rows += c->h_lens[b];
+    for (int b = 0; b < batch; ++b)
+        rows += c->h_lens[b] < c->cfg.max_seq ? c->h_lens[b] : c->cfg.max_seq;
     const double bytes = (double)rows * 4.0 * c->cfg.n_kv_heads * c->cfg.head_dim;
     if (bytes <= 0 || c->l2_keep_bytes <= 0) return 0.f;
     const double f = std::fmin(1.0, c->l2_keep_bytes / bytes);
@@ -570,7 +575,7 @@ int lckv_cache_reset(lckv_cache_t* c, const int32_t* host_lens, int32_t batch, v
     if (host_lens) {
         for (int b = 0; b < batch; ++b) {
             if (host_lens[b] < 0) return LCKV_EINVAL;
-            if (host_lens[b] > c->cfg.max_seq) return LCKV_ECAPACITY;
+            if (host_lens[b] > c->cfg.max_seq && c->cfg.stream_sink == 0) return LCKV_ECAPACITY;
         }
         for (int b = 0; b < batch; ++b) c->h_lens[b] = host_lens[b];
         // h_lens is the staging source: it lives as long as the cache and pageable copies are
@@ -775,7 +780,8 @@ extern "C" int lckv_decode_attention_static(const void* k, const void* v, const 
     if (!k || !v || !lens || !q || !out) return LCKV_EINVAL;
     if (batch < 1 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads) return LCKV_EINVAL;
     if (head_dim != 64 && head_dim != 128) return LCKV_EINVAL;
-    if (max_seq < 1 || (mode != LCKV_MODE_CONDENSED && mode != LCKV_MODE_STANDARD)) return LCKV_EINVAL;
+    if (max_seq < 1 || max_seq > 0x7fffffff) return LCKV_EINVAL;
+    if (mode != LCKV_MODE_CONDENSED && mode != LCKV_MODE_STANDARD) return LCKV_EINVAL;
     if (out_dtype != 0 && out_dtype != 1) return LCKV_EINVAL;
     if (!(softmax_scale >= 0.f) || !std::isfinite(softmax_scale)) return LCKV_EINVAL;
     if (batch > LCKV_STATIC_MAX_BATCH) return LCKV_ESTATICLIMIT;
@@ -801,7 +807,7 @@ extern "C" int lckv_decode_attention_static(const void* k, const void* v, const 
 
     const int R = lckv::kAluSlotBytes / (head_dim * 2);
     lckv::plan_kernel<<<1, 1024, 0, st>>>(lens, batch, R, n_q_heads, n_workers, d_pre,
-                                          kStaticPreStride, d_start);
+                                          kStaticPreStride, d_start, (int)max_seq);
     if (!cuda_ok(cudaGetLastError())) return LCKV_ECUDA;
 
     lckv::AttnParams p;

@@ -65,7 +65,7 @@ struct TileCursor {
 __device__ __forceinline__ void cursor_load(TileCursor& c, const AttnParams& p)
 {
     c.nt = __ldg(p.pre + c.b + 1) - __ldg(p.pre + c.b);
-    c.nv = __ldg(p.lens + c.b) + p.mode;
+    c.nv = min(__ldg(p.lens + c.b) + p.mode, (int32_t)p.T_cap);  // a cache holds at most T_cap rows
 }
 
 // Next tile in (b, pair, tile) order, skipping sequences without tiles.  Safe past the end.

@@ -84,7 +84,7 @@ struct RowCursor {
 __device__ __forceinline__ void rcursor_load(RowCursor& c, const AttnParams& p)
 {
     c.nt = __ldg(p.pre + c.b + 1) - __ldg(p.pre + c.b);
-    c.nv = __ldg(p.lens + c.b) + p.mode;
+    c.nv = min(__ldg(p.lens + c.b) + p.mode, (int32_t)p.T_cap);  // a cache holds at most T_cap rows
 }
 
 // After b, h, t are set: derive the kv head and the tile's first row.  per_kv = pairs per kv head.

@@ -11,11 +11,12 @@ namespace lckv {
 // This kernel (one block) writes, for both mask modes (n_vis = len + mode):
 //   pre[mode][b]      tiles of sequences 0..b-1 (exclusive prefix; pre[mode][B] = all tiles / H)
 //   start_b[mode][w]  the sequence in which worker w's range begins
-// so an attention worker needs two small loads to find its place.
+// so an attention worker needs two small loads to find its place.  n_vis is capped at T_cap: in
+// streaming mode (sink + recent window) a cache never holds more than T_cap rows.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024)
 plan_kernel(const int32_t* __restrict__ lens, int B, int R, int H, int n_workers,
-            uint32_t* pre, int pre_stride, int32_t* __restrict__ start_b)
+            uint32_t* pre, int pre_stride, int32_t* __restrict__ start_b, int T_cap)
 {
     __shared__ uint32_t warp_sums[32];
     __shared__ uint32_t carry;
@@ -26,7 +27,7 @@ plan_kernel(const int32_t* __restrict__ lens, int B, int R, int H, int n_workers
         uint32_t* pr = pre + mode * pre_stride;
         const int b0 = min(B, tid * chunk), b1 = min(B, b0 + chunk);
         uint32_t local = 0;
-        for (int b = b0; b < b1; ++b) local += (uint32_t)(lens[b] + mode + R - 1) / (uint32_t)R;
+        for (int b = b0; b < b1; ++b) local += (uint32_t)(min(lens[b] + mode, T_cap) + R - 1) / (uint32_t)R;
         // block-wide exclusive scan of `local`
         uint32_t incl = local;
         for (int off = 1; off < 32; off <<= 1) {
@@ -48,7 +49,7 @@ plan_kernel(const int32_t* __restrict__ lens, int B, int R, int H, int n_workers
         uint32_t run = warp_sums[warp] + incl - local;
         for (int b = b0; b < b1; ++b) {
             pr[b] = run;
-            run += (uint32_t)(lens[b] + mode + R - 1) / (uint32_t)R;
+            run += (uint32_t)(min(lens[b] + mode, T_cap) + R - 1) / (uint32_t)R;
         }
         if (tid == 0) pr[B] = carry;
         __syncthreads();  // pr[] (global) is now visible to the whole block
@@ -75,11 +76,13 @@ plan_kernel(const int32_t* __restrict__ lens, int B, int R, int H, int n_workers
 }
 
 // Row len[b] of K and V <- k_new, v_new (bit-exact 16-byte copies).  One thread per 16 bytes.
+// With n_sink > 0 (StreamingLLM-style cache, paper Section 3.3) token t >= T_cap replaces the oldest
+// non-sink token: row n_sink + (t - n_sink) mod (T_cap - n_sink).
 __global__ void append_kernel(uint16_t* __restrict__ K, uint16_t* __restrict__ V,
                               const uint16_t* __restrict__ k_new,
                               const uint16_t* __restrict__ v_new,
                               const int32_t* __restrict__ lens, int B, int H_kv, int64_t T_cap,
-                              int D)
+                              int D, int n_sink)
 {
     const int chunks = D / 8;
     const int64_t n = (int64_t)B * H_kv * chunks;
@@ -88,7 +91,9 @@ __global__ void append_kernel(uint16_t* __restrict__ K, uint16_t* __restrict__ V
     const int c = (int)(i % chunks);
     const int64_t bh = i / chunks;
     const int b = (int)(bh / H_kv);
-    const int64_t row = lens[b];
+    int64_t row = lens[b];
+    // Streaming mode: the first n_sink rows stay, the others form a ring of the most recent tokens.
+    if (n_sink > 0 && row >= T_cap) row = n_sink + (row - n_sink) % (T_cap - n_sink);
     if (row < 0 || row >= T_cap) return;  // the host refuses such calls; never write out of range
     const int64_t dst = (bh * T_cap + row) * D + c * 8;
     const int64_t src = bh * D + c * 8;

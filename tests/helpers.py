@@ -38,7 +38,8 @@ class Case:
     """One layer stack with GPU cache and host (oracle) caches holding the same bits."""
 
     def __init__(self, L, w, Hq, Hkv, d, lens, T_cap, variant=0, out_dtype=0, seed=1234, std=1.0,
-                 poison=True, B_max=None, scale=0.0, kernel_kind=0, host_staging=0, use_graph=0):
+                 poison=True, B_max=None, scale=0.0, kernel_kind=0, host_staging=0, use_graph=0,
+                 stream_sink=0):
         self.L, self.w, self.Hq, self.Hkv, self.d = L, w, Hq, Hkv, d
         self.lens = np.asarray(lens, np.int32).copy()
         self.B = len(lens)
@@ -46,7 +47,9 @@ class Case:
         B_max = B_max or self.B
         self.cfg = lk.make_config(L, w, Hq, Hkv, d, B_max, T_cap, softmax_scale=scale,
                                   top_variant=variant, out_dtype=out_dtype, kernel_kind=kernel_kind,
-                                  host_staging=host_staging, use_graph=use_graph)
+                                  host_staging=host_staging, use_graph=use_graph,
+                                  stream_sink=stream_sink)
+        self.stream_sink = stream_sink
         self.scale = scale if scale > 0 else d ** -0.5
         self.cache = lk.Cache(self.cfg)
         self.plan = orc.plan(L, w, variant)
@@ -58,7 +61,7 @@ class Case:
             vb = syn.bits(syn.randn_bf16((B_max, Hkv, T_cap, d), seed + 2 * s + 1, std=std))
             if poison:
                 for b in range(B_max):
-                    n = int(self.lens[b]) if b < self.B else 0
+                    n = min(int(self.lens[b]), T_cap) if b < self.B else 0
                     kb[b, :, n:] = NAN_BITS
                     vb[b, :, n:] = NAN_BITS
             kt, vt = self.cache.slot_tensors(s)
@@ -98,7 +101,8 @@ class Case:
         want, _ = orc.stack_step(self.L, self.w, [syn.bits(t) for t in q],
                                  [None if t is None else syn.bits(t) for t in kn],
                                  [None if t is None else syn.bits(t) for t in vn],
-                                 self.hK, self.hV, self.lens, self.scale, top_variant=self.variant)
+                                 self.hK, self.hV, self.lens, self.scale, top_variant=self.variant,
+                                 n_sink=self.stream_sink)
         self.step_no += 1
         stats = []
         if check:

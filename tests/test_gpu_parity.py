@@ -254,3 +254,16 @@ def test_graph_replay_steps_match(shape):
     c.close()
     torch.cuda.synchronize()
     torch.cuda.set_stream(torch.cuda.default_stream())
+
+
+@pytest.mark.parametrize("shape", ["mha", "gqa"])
+def test_streaming_sink_and_window_cache(shape):
+    """StreamingLLM-style caches (4 sinks + recent window): decode across the point where the ring
+    wraps, some sequences already far past the capacity; outputs, ring rows and lengths exact."""
+    kw = dict(Hq=4, Hkv=4, d=128, std=1.0) if shape == "mha" else dict(Hq=16, Hkv=2, d=64, std=0.25)
+    T_cap = 37
+    c = Case(L=4, w=2, lens=[0, 30, 35, 36, 37, 38, 100, 5000], T_cap=T_cap, seed=91, stream_sink=4, **kw)
+    for _ in range(8):
+        c.step()
+    assert c.lens.tolist() == [8, 38, 43, 44, 45, 46, 108, 5008]
+    c.close()

@@ -366,3 +366,53 @@ def test_golden_two_key_example():
         o, lse = orc.attend_row(q, K[:int(n_vis)], V[:int(n_vis)], 1.0)
         np.testing.assert_allclose(o[0], float(want_o), atol=1e-15)
         np.testing.assert_allclose(lse, float(want_lse), atol=1e-15)
+
+
+# ---- sink + recent-window caches (Section 3.3: integration with StreamingLLM) ---------------------
+
+def test_streaming_ring_rows_enumerated_by_hand():
+    """Cache of 6 rows with 2 sinks: tokens 0..5 fill rows 0..5, then the 4 non-sink rows are reused
+    in turn.  Written out by hand."""
+    C_, s = 6, 2
+    want_rows = [0, 1, 2, 3, 4, 5, 2, 3, 4, 5, 2, 3]
+    K = np.zeros((1, 1, C_, 4), np.uint16); V = np.zeros_like(K)
+    for t, row in enumerate(want_rows):
+        k = np.full((1, 1, 4), 100 + t, np.uint16)
+        before = K.copy()
+        orc.append(K, V, k, k, np.array([t], np.int32), n_sink=s)
+        changed = np.nonzero((K != before).any(axis=-1)[0, 0])[0].tolist()
+        assert changed == [row], (t, changed)
+        assert (K[0, 0, row] == 100 + t).all()
+
+
+@pytest.mark.parametrize("w", [0, 1])
+def test_streaming_equals_attention_over_sinks_plus_recent_tokens(w):
+    """Decode n tokens through a small ring cache; each output must equal plain attention, computed
+    here from the full history, over the first s tokens plus the most recent C - s tokens that the
+    query may see (before t for the diagonal-masked layers, up to and including t for standard
+    layers).  Row order inside the ring is irrelevant (permutation invariance)."""
+    n, d, C_, s = 25, 8, 9, 3
+    qb, kb, vb = rand_bits((n, 1, 1, d), 71), rand_bits((n, 1, 1, d), 72), rand_bits((n, 1, 1, d), 73)
+    K = np.zeros((1, 1, C_, d), np.uint16); V = np.zeros_like(K)
+    lens = np.zeros(1, np.int32)
+    Kh, Vh, Q = f64(kb[:, 0, 0]), f64(vb[:, 0, 0]), f64(qb[:, 0, 0])
+    for t in range(n):
+        outs, _ = orc.stack_step(1, w, [qb[t]], [kb[t]], [vb[t]], [K], [V], lens, 0.4, n_sink=s)
+        last = t + 1 if w else t                      # exclusive end of what the query may see
+        vis = list(range(min(s, last))) + list(range(max(s, last - (C_ - s)), last))
+        if not vis:
+            assert not outs[0].any()
+            continue
+        sc = 0.4 * (Kh[vis] @ Q[t]); p = np.exp(sc - sc.max()); p /= p.sum()
+        np.testing.assert_allclose(outs[0][0, 0], p @ Vh[vis], atol=1e-12)
+    assert lens[0] == n
+    # until the cache is full the policy changes nothing
+    K2 = np.zeros((1, 1, C_, d), np.uint16); V2 = np.zeros_like(K2); l2 = np.zeros(1, np.int32)
+    K3 = K2.copy(); V3 = V2.copy(); l3 = np.zeros(1, np.int32)
+    for t in range(C_):
+        a, _ = orc.stack_step(1, w, [qb[t]], [kb[t]], [vb[t]], [K2], [V2], l2, 0.4, n_sink=s)
+        b, _ = orc.stack_step(1, w, [qb[t]], [kb[t]], [vb[t]], [K3], [V3], l3, 0.4)
+        assert np.array_equal(a[0], b[0])
+    assert np.array_equal(K2, K3)
+    with pytest.raises(orc.OracleError):   # without the policy the 10th token does not fit
+        orc.stack_step(1, w, [qb[C_]], [kb[C_]], [vb[C_]], [K3], [V3], l3, 0.4)
