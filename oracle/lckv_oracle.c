@@ -295,3 +295,108 @@ int lckv_oracle_num_threads(void)
 #endif
     return n;
 }
+
+/* ------------------------------------------------------------------------------------------------
+ * Prompt encoding (Section 2.3 "Inference with Prompts"; Section 2.2.1 for one parallel iteration).
+ *
+ * The prompt cannot be encoded in one parallel pass, because every token needs the top-layer k,v
+ * of its predecessors.  Instead the paper runs m + b iterations over all prompt tokens in parallel;
+ * in each iteration the queries of the condensed layers are paired with the top-layer k,v of the
+ * PREVIOUS iteration (zero vectors before the first one), diagonal masked as always, and the
+ * warmup layers do standard causal attention over their own k,v of the current iteration.
+ *
+ * Token-parallel attention of one layer:
+ *   q    [B, n_max, H_q, d]   token-major; tokens i < lens[b] of sequence b are valid
+ *   K, V [B, H_kv, T_cap, d]  cache; rows j < lens[b] valid
+ *   mode 0: token i sees rows j < i;  mode 1: rows j <= i
+ *   out  [B, n_max, H_q, d] float64; rows i >= lens[b] are left untouched
+ * Each (b, i, h) is one attend_row call: the definition, nothing shared with the decode path's
+ * bookkeeping.
+ * ------------------------------------------------------------------------------------------------ */
+int lckv_oracle_prefill_attention(const uint16_t* q, const uint16_t* K, const uint16_t* V,
+                                  const int32_t* lens, int B, int n_max, int H_q, int H_kv,
+                                  int64_t T_cap, int d, int mode, double scale, int always_sink,
+                                  double* out)
+{
+    if (B < 0 || n_max < 0 || H_q < 1 || H_kv < 1 || H_q % H_kv != 0 || d < 1) return LCKV_ORACLE_EINVAL;
+    if (mode != 0 && mode != 1) return LCKV_ORACLE_EINVAL;
+    int g = H_q / H_kv;
+    for (int b = 0; b < B; ++b)
+        if (lens[b] < 0 || lens[b] > n_max || (int64_t)lens[b] > T_cap) return LCKV_ORACLE_ECAPACITY;
+    int64_t rows = (int64_t)B * n_max * H_q;
+#pragma omp parallel
+    {
+        double* scratch = (double*)malloc(sizeof(double) * (size_t)(n_max > 0 ? n_max : 1));
+#pragma omp for schedule(dynamic, 16)
+        for (int64_t r = 0; r < rows; ++r) {
+            int h = (int)(r % H_q);
+            int i = (int)((r / H_q) % n_max);
+            int b = (int)(r / ((int64_t)H_q * n_max));
+            if (i >= lens[b]) continue;
+            int kvh = h / g;
+            int64_t n_vis = (int64_t)i + mode;
+            const uint16_t* Kp = K + (((int64_t)b * H_kv + kvh) * T_cap) * d;
+            const uint16_t* Vp = V + (((int64_t)b * H_kv + kvh) * T_cap) * d;
+            attend_row(q + r * d, Kp, Vp, n_vis, d, scale, always_sink, out + r * d, NULL, NULL,
+                       scratch);
+        }
+        free(scratch);
+    }
+    return LCKV_ORACLE_OK;
+}
+
+/* Rows [0, lens[b]) of a cache <- the prompt's k, v ([B, n_max, H_kv, d], token-major). */
+int lckv_oracle_prefill_write_kv(uint16_t* K, uint16_t* V, const uint16_t* k, const uint16_t* v,
+                                 const int32_t* lens, int B, int n_max, int H_kv, int64_t T_cap,
+                                 int d)
+{
+    for (int b = 0; b < B; ++b)
+        if (lens[b] < 0 || lens[b] > n_max || (int64_t)lens[b] > T_cap) return LCKV_ORACLE_ECAPACITY;
+    for (int b = 0; b < B; ++b)
+        for (int i = 0; i < lens[b]; ++i)
+            for (int h = 0; h < H_kv; ++h) {
+                int64_t dst = ((((int64_t)b * H_kv + h) * T_cap) + i) * d;
+                int64_t src = (((int64_t)b * n_max + i) * H_kv + h) * d;
+                memcpy(K + dst, k + src, sizeof(uint16_t) * (size_t)d);
+                memcpy(V + dst, v + src, sizeof(uint16_t) * (size_t)d);
+            }
+    return LCKV_ORACLE_OK;
+}
+
+/*
+ * One parallel iteration over the whole layer stack (Section 2.2.1 / 2.3), following the same
+ * layer plan as a decode step: a warmup layer first stores its k,v of this iteration in its own
+ * cache and then attends causally (j <= i); a condensed layer attends j < i over the shared
+ * cache, which still holds the previous iteration's top-layer k,v; at the end of the iteration the
+ * feeder layer's k,v of this iteration replace them.  Lengths do not change.
+ */
+int lckv_oracle_prefill_iteration(int L, int w, int top_variant, const uint16_t* const* q_layers,
+                                  const uint16_t* const* k_layers, const uint16_t* const* v_layers,
+                                  uint16_t* const* K_slots, uint16_t* const* V_slots,
+                                  const int32_t* lens, int B, int n_max, int H_q, int H_kv,
+                                  int64_t T_cap, int d, double scale, int always_sink,
+                                  double* const* out_layers)
+{
+    int32_t* plan = (int32_t*)malloc(sizeof(int32_t) * 5 * (size_t)L);
+    if (!plan) return LCKV_ORACLE_EINVAL;
+    int32_t *is_w = plan, *rs = plan + L, *md = plan + 2 * L, *ws = plan + 3 * L, *wb = plan + 4 * L;
+    int32_t n_slots = 0;
+    int rc = lckv_oracle_plan(L, w, top_variant, is_w, rs, md, ws, wb, &n_slots);
+    for (int l = 0; l < L && rc == 0; ++l)
+        if (ws[l] >= 0 && (!k_layers[l] || !v_layers[l])) rc = LCKV_ORACLE_EINVAL;
+    for (int l = 0; l < L && rc == 0; ++l) {
+        if (ws[l] >= 0 && wb[l])
+            rc = lckv_oracle_prefill_write_kv(K_slots[ws[l]], V_slots[ws[l]], k_layers[l],
+                                              v_layers[l], lens, B, n_max, H_kv, T_cap, d);
+        if (rc) break;
+        rc = lckv_oracle_prefill_attention(q_layers[l], K_slots[rs[l]], V_slots[rs[l]], lens, B,
+                                           n_max, H_q, H_kv, T_cap, d, md[l], scale, always_sink,
+                                           out_layers[l]);
+    }
+    for (int l = 0; l < L && rc == 0; ++l)
+        if (ws[l] >= 0 && !wb[l])
+            rc = lckv_oracle_prefill_write_kv(K_slots[ws[l]], V_slots[ws[l]], k_layers[l],
+                                              v_layers[l], lens, B, n_max, H_kv, T_cap, d);
+    free(plan);
+    return rc;
+}

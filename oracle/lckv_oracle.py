@@ -39,6 +39,17 @@ def lib():
                                              C.c_int, C.c_int, C.c_int, C.c_int64, C.c_int,
                                              C.c_double, C.c_int, C.c_int, pp, pp]
         L.lckv_oracle_stack_step.restype = C.c_int
+        L.lckv_oracle_prefill_attention.argtypes = [u16p, u16p, u16p, i32p, C.c_int, C.c_int,
+                                                    C.c_int, C.c_int, C.c_int64, C.c_int, C.c_int,
+                                                    C.c_double, C.c_int, f64p]
+        L.lckv_oracle_prefill_attention.restype = C.c_int
+        L.lckv_oracle_prefill_write_kv.argtypes = [u16p, u16p, u16p, u16p, i32p, C.c_int, C.c_int,
+                                                   C.c_int, C.c_int64, C.c_int]
+        L.lckv_oracle_prefill_write_kv.restype = C.c_int
+        L.lckv_oracle_prefill_iteration.argtypes = [C.c_int, C.c_int, C.c_int, pp, pp, pp, pp, pp,
+                                                    i32p, C.c_int, C.c_int, C.c_int, C.c_int,
+                                                    C.c_int64, C.c_int, C.c_double, C.c_int, pp]
+        L.lckv_oracle_prefill_iteration.restype = C.c_int
         L.lckv_oracle_num_threads.restype = C.c_int
         _LIB = L
     return _LIB
@@ -157,3 +168,54 @@ def stack_step(L, w, q_layers, k_new_layers, v_new_layers, K_slots, V_slots, len
                                       _ptr_array(lses))
     _chk(rc, "stack_step")
     return outs, lses
+
+
+def prefill_attention(q, K, V, lens, mode, scale, always_sink=False):
+    """Token-parallel attention of one layer (prompt encoding, Section 2.3).
+    q [B,n_max,Hq,d], K,V [B,Hkv,Tcap,d] uint16, lens [B] -> out [B,n_max,Hq,d] float64
+    (rows i >= lens[b] are zero)."""
+    q, K, V = _u16(q), _u16(K), _u16(V)
+    lens = np.ascontiguousarray(lens, np.int32)
+    B, n_max, Hq, d = q.shape
+    _, Hkv, Tcap, _ = K.shape
+    out = np.zeros((B, n_max, Hq, d), np.float64)
+    rc = lib().lckv_oracle_prefill_attention(_p(q, C.c_uint16), _p(K, C.c_uint16),
+                                             _p(V, C.c_uint16), _p(lens, C.c_int32), B, n_max, Hq,
+                                             Hkv, Tcap, d, int(mode), float(scale),
+                                             int(always_sink), _p(out, C.c_double))
+    _chk(rc, "prefill_attention")
+    return out
+
+
+def prefill_write_kv(K, V, k, v, lens):
+    """In place: rows [0, lens[b]) of K,V [B,Hkv,Tcap,d] <- k, v [B,n_max,Hkv,d]."""
+    assert K.flags.c_contiguous and V.flags.c_contiguous and K.dtype == np.uint16
+    k, v = _u16(k), _u16(v)
+    lens = np.ascontiguousarray(lens, np.int32)
+    B, n_max, Hkv, d = k.shape
+    rc = lib().lckv_oracle_prefill_write_kv(_p(K, C.c_uint16), _p(V, C.c_uint16),
+                                            _p(k, C.c_uint16), _p(v, C.c_uint16),
+                                            _p(lens, C.c_int32), B, n_max, Hkv, K.shape[2], d)
+    _chk(rc, "prefill_write_kv")
+
+
+def prefill_iteration(L, w, q_layers, k_layers, v_layers, K_slots, V_slots, lens, scale,
+                      top_variant=0, always_sink=False):
+    """One parallel iteration over the stack; caches updated in place.  Returns the list of L
+    outputs [B,n_max,Hq,d] float64."""
+    q_layers = [_u16(q) for q in q_layers]
+    k_layers = [None if k is None else _u16(k) for k in k_layers]
+    v_layers = [None if v is None else _u16(v) for v in v_layers]
+    for a in list(K_slots) + list(V_slots):
+        assert a.flags.c_contiguous and a.dtype == np.uint16
+    lens = np.ascontiguousarray(lens, np.int32)
+    B, n_max, Hq, d = q_layers[0].shape
+    _, Hkv, Tcap, _ = K_slots[0].shape
+    outs = [np.zeros((B, n_max, Hq, d), np.float64) for _ in range(L)]
+    rc = lib().lckv_oracle_prefill_iteration(L, w, int(top_variant), _ptr_array(q_layers),
+                                             _ptr_array(k_layers), _ptr_array(v_layers),
+                                             _ptr_array(K_slots), _ptr_array(V_slots),
+                                             _p(lens, C.c_int32), B, n_max, Hq, Hkv, Tcap, d,
+                                             float(scale), int(always_sink), _ptr_array(outs))
+    _chk(rc, "prefill_iteration")
+    return outs
