@@ -232,6 +232,42 @@ int lckv_layer_stack_step_host(lckv_cache_t* cache, const void* const* q_layers_
                                void* stream);
 
 /*
+ * Prompt encoding (Section 2.3: the prompt is encoded by m + b parallel
+ * iterations; Section 2.2.1 defines one iteration: all tokens in parallel, the
+ * condensed layers paired with the top-layer k,v of the PREVIOUS iteration -
+ * zero vectors before the first one - and the diagonal masked).  These calls
+ * are the attention and cache-write operations of one such iteration.  They
+ * require lengths already set to the prompt lengths (lckv_cache_reset) and do
+ * not change them; n_max >= every len[b] of the batch is the token stride of
+ * the token-major tensors.  Not available with stream_sink > 0.
+ *
+ * lckv_prefill_write_kv: rows [0, len[b]) of slot `slot` <- k, v
+ *   [batch, n_max, H_kv, d_h] bf16 (bit-exact copies; other rows untouched).
+ * lckv_prefill_attention: for every token i < len[b] and head h,
+ *   out[b,i,h] = softmax-weighted sum over rows j < i (LCKV_MODE_CONDENSED) or
+ *   j <= i (LCKV_MODE_STANDARD) of the slot; a token that sees nothing gets
+ *   the zero vector.  q, out: [batch, n_max, H_q, d_h] (out bf16 or fp32 per
+ *   out_dtype); rows i >= len[b] of out are not written.  Tensor-core kernel,
+ *   fp32 accumulation, probabilities rounded to bf16 for the second product.
+ * lckv_prefill_iteration: one iteration over the whole stack in plan order
+ *   (write_before layers store their k,v and attend causally; condensed layers
+ *   attend slot 0, which still holds the previous iteration's top-layer k,v;
+ *   at the end the feeder layer's k,v replace them).  Before the first
+ *   iteration the caller zero-fills slot 0 (the dummy zero k,v).  Array
+ *   arguments as in lckv_layer_stack_step, tensors token-major as above.
+ * Errors: EINVAL (null, bad slot/mode/batch, n_max < 1, a len[b] > n_max,
+ * stream_sink > 0), ECUDA.
+ */
+int lckv_prefill_write_kv(lckv_cache_t* cache, int32_t slot, const void* k, const void* v,
+                          int32_t n_max, int32_t batch, void* stream);
+int lckv_prefill_attention(lckv_cache_t* cache, int32_t slot, int32_t mode, const void* q,
+                           void* out, int32_t n_max, int32_t batch, void* stream);
+int lckv_prefill_iteration(lckv_cache_t* cache, const void* const* q_layers,
+                           void* const* out_layers, const void* const* k_layers,
+                           const void* const* v_layers, int32_t n_max, int32_t batch,
+                           void* stream);
+
+/*
  * Decode attention without a cache object and without any allocation (the
  * paper has no counterpart: this is a packaging variant of
  * lckv_decode_attention for callers that cannot allocate).

@@ -47,6 +47,9 @@ SIGNATURES = {
     "lckv_decode_attention": (C.c_int, [_vp, _i32, _i32, _vp, _vp, _vp, _i32, _vp]),
     "lckv_layer_stack_step": (C.c_int, [_vp, _vpp, _vpp, _vpp, _vpp, _i32, _vp]),
     "lckv_layer_stack_step_host": (C.c_int, [_vp, _vpp, _vpp, _vpp, _vpp, _i32, _vp]),
+    "lckv_prefill_write_kv": (C.c_int, [_vp, _i32, _vp, _vp, _i32, _i32, _vp]),
+    "lckv_prefill_attention": (C.c_int, [_vp, _i32, _i32, _vp, _vp, _i32, _i32, _vp]),
+    "lckv_prefill_iteration": (C.c_int, [_vp, _vpp, _vpp, _vpp, _vpp, _i32, _i32, _vp]),
     "lckv_decode_attention_static": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32,
                                               _i32, C.c_int64, _i32, C.c_float, _i32, _vp]),
     "lckv_status_string": (C.c_char_p, [C.c_int]),
@@ -237,3 +240,21 @@ class Cache:
                                               _ptr_array(out_layers), _ptr_array(k_new_layers),
                                               _ptr_array(v_new_layers), batch, _stream(stream)),
              "lckv_layer_stack_step_host")
+
+    # -- prompt encoding (token-major tensors [B, n_max, H, d_h]) -------------------------------
+    def lckv_prefill_write_kv(self, slot, k, v, stream=None):
+        _chk(lib().lckv_prefill_write_kv(self.h, slot, _ptr(k), _ptr(v), k.shape[1], k.shape[0],
+                                         _stream(stream)), "lckv_prefill_write_kv")
+
+    def lckv_prefill_attention(self, slot, mode, q, out=None, stream=None):
+        if out is None:
+            out = torch.zeros(q.shape, dtype=self.out_torch_dtype, device=q.device)
+        _chk(lib().lckv_prefill_attention(self.h, slot, mode, _ptr(q), _ptr(out), q.shape[1],
+                                          q.shape[0], _stream(stream)), "lckv_prefill_attention")
+        return out
+
+    def lckv_prefill_iteration(self, q_layers, out_layers, k_layers, v_layers, stream=None):
+        q0 = q_layers[0]
+        _chk(lib().lckv_prefill_iteration(self.h, _ptr_array(q_layers), _ptr_array(out_layers),
+                                          _ptr_array(k_layers), _ptr_array(v_layers), q0.shape[1],
+                                          q0.shape[0], _stream(stream)), "lckv_prefill_iteration")

@@ -11,6 +11,7 @@
 #include "../../include/lckv.h"
 #include "lckv_attn_alu.cuh"
 #include "lckv_attn_mma.cuh"
+#include "lckv_prefill.cuh"
 #include "lckv_small_kernels.cuh"
 
 namespace {
@@ -89,6 +90,7 @@ struct lckv_cache {
     std::vector<int32_t> h_lens;  // host mirror of the device lengths
     int n_kv_layers;
     std::vector<CUtensorMap> tm_k, tm_v;  // per slot, tensor-core kernel only
+    std::vector<CUtensorMap> tm_pf_k, tm_pf_v;  // per slot, 64-row boxes for prompt encoding
     double l2_keep_bytes;                 // how much of a re-read slot to hold in L2 (0 = off)
     int ws_parity;                        // which half of the split-K workspace the next launch uses
     size_t partials_half_floats;          // floats in one half of the partial records
@@ -434,6 +436,56 @@ int run_step(lckv_cache* c, const void* const* q, void* const* out, const void* 
     return rc;
 }
 
+int prefill_check(const lckv_cache* c, int n_max, int batch)
+{
+    if (c->cfg.stream_sink > 0 || c->tm_pf_k.empty()) return LCKV_EINVAL;
+    if (batch < 1 || batch > c->cfg.max_batch || n_max < 1) return LCKV_EINVAL;
+    for (int b = 0; b < batch; ++b)
+        if (c->h_lens[b] > n_max) return LCKV_EINVAL;
+    return LCKV_OK;
+}
+
+int launch_prefill_write(lckv_cache* c, int slot, const void* k, const void* v, int n_max,
+                         int batch, cudaStream_t st)
+{
+    const int64_t n = (int64_t)batch * n_max * c->cfg.n_kv_heads * (c->cfg.head_dim / 8);
+    const int threads = 256;
+    lckv::prefill_write_kv_kernel<<<(unsigned)((n + threads - 1) / threads), threads, 0, st>>>(
+        slot_k(c, slot), slot_v(c, slot), static_cast<const uint16_t*>(k),
+        static_cast<const uint16_t*>(v), c->d_lens, batch, n_max, c->cfg.n_kv_heads, c->cfg.max_seq,
+        c->cfg.head_dim);
+    return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
+}
+
+int launch_prefill_attention(lckv_cache* c, int slot, int mode, const void* q, void* out,
+                             int n_max, int batch, cudaStream_t st)
+{
+    lckv::PrefillParams p;
+    p.q = static_cast<const uint16_t*>(q);
+    p.out = out;
+    p.lens = c->d_lens;
+    p.status = c->d_status;
+    p.T_cap = c->cfg.max_seq;
+    p.B = batch;
+    p.n_max = n_max;
+    p.H_q = c->cfg.n_q_heads;
+    p.H_kv = c->cfg.n_kv_heads;
+    p.mode = mode;
+    p.out_f32 = c->cfg.out_dtype;
+    p.scale_log2 = c->scale_log2;
+    int longest = 0;
+    for (int b = 0; b < batch; ++b) longest = c->h_lens[b] > longest ? c->h_lens[b] : longest;
+    if (longest == 0) return LCKV_OK;
+    const dim3 grid((longest + lckv::kPfBM - 1) / lckv::kPfBM, c->cfg.n_q_heads, batch);
+    if (c->cfg.head_dim == 128)
+        lckv::prefill_attn_kernel<128><<<grid, lckv::kPfWarps * 32, lckv::prefill_smem_bytes<128>(), st>>>(
+            p, c->tm_pf_k[slot], c->tm_pf_v[slot]);
+    else
+        lckv::prefill_attn_kernel<64><<<grid, lckv::kPfWarps * 32, lckv::prefill_smem_bytes<64>(), st>>>(
+            p, c->tm_pf_k[slot], c->tm_pf_v[slot]);
+    return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
+}
+
 }  // namespace
 
 extern "C" {
@@ -526,7 +578,26 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
             if (rc) { delete c; return rc; }
         }
     }
-    bool ok = cuda_ok(cudaFuncSetAttribute(lckv::attn_mma_kernel<128>,
+    {
+        // prompt-encoding kernel: 64-row boxes over every slot (coordinates are 32-bit)
+        const uint64_t rows = (uint64_t)cfg->max_batch * cfg->n_kv_heads * (uint64_t)cfg->max_seq;
+        if (rows < (1ull << 31)) {
+            c->tm_pf_k.resize(c->plan.n_slots);
+            c->tm_pf_v.resize(c->plan.n_slots);
+            for (int s = 0; s < c->plan.n_slots; ++s) {
+                int rc = make_tensor_map(&c->tm_pf_k[s], slot_k(c, s), rows, cfg->head_dim, lckv::kPfBN);
+                if (!rc) rc = make_tensor_map(&c->tm_pf_v[s], slot_v(c, s), rows, cfg->head_dim, lckv::kPfBN);
+                if (rc) { delete c; return rc; }
+            }
+        }
+    }
+    bool ok = cuda_ok(cudaFuncSetAttribute(lckv::prefill_attn_kernel<128>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           lckv::prefill_smem_bytes<128>())) &&
+              cuda_ok(cudaFuncSetAttribute(lckv::prefill_attn_kernel<64>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           lckv::prefill_smem_bytes<64>())) &&
+              cuda_ok(cudaFuncSetAttribute(lckv::attn_mma_kernel<128>,
                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            lckv::kMmaSmemBytes)) &&
               cuda_ok(cudaFuncSetAttribute(lckv::attn_mma_kernel<64>,
@@ -702,6 +773,52 @@ int lckv_layer_stack_step_host(lckv_cache_t* c, const void* const* q_host, void*
     for (int l = 0; l < L; ++l)
         if (!cuda_ok(cudaMemcpyAsync(out_host[l], dout[l], o_bytes, cudaMemcpyDeviceToHost, st)))
             return LCKV_ECUDA;
+    return LCKV_OK;
+}
+
+int lckv_prefill_write_kv(lckv_cache_t* c, int32_t slot, const void* k, const void* v,
+                          int32_t n_max, int32_t batch, void* stream)
+{
+    if (!c || !k || !v || slot < 0 || slot >= c->plan.n_slots) return LCKV_EINVAL;
+    if (int rc = prefill_check(c, n_max, batch)) return rc;
+    return launch_prefill_write(c, slot, k, v, n_max, batch, static_cast<cudaStream_t>(stream));
+}
+
+int lckv_prefill_attention(lckv_cache_t* c, int32_t slot, int32_t mode, const void* q, void* out,
+                           int32_t n_max, int32_t batch, void* stream)
+{
+    if (!c || !q || !out || slot < 0 || slot >= c->plan.n_slots) return LCKV_EINVAL;
+    if (mode != LCKV_MODE_CONDENSED && mode != LCKV_MODE_STANDARD) return LCKV_EINVAL;
+    if (int rc = prefill_check(c, n_max, batch)) return rc;
+    return launch_prefill_attention(c, slot, mode, q, out, n_max, batch,
+                                    static_cast<cudaStream_t>(stream));
+}
+
+int lckv_prefill_iteration(lckv_cache_t* c, const void* const* q_layers, void* const* out_layers,
+                           const void* const* k_layers, const void* const* v_layers, int32_t n_max,
+                           int32_t batch, void* stream)
+{
+    if (!c || !q_layers || !out_layers || !k_layers || !v_layers) return LCKV_EINVAL;
+    if (int rc = prefill_check(c, n_max, batch)) return rc;
+    const Plan& pl = c->plan;
+    const int L = c->cfg.n_layers;
+    for (int l = 0; l < L; ++l) {
+        if (!q_layers[l] || !out_layers[l]) return LCKV_EINVAL;
+        if (pl.write_slot[l] >= 0 && (!k_layers[l] || !v_layers[l])) return LCKV_EINVAL;
+    }
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    for (int l = 0; l < L; ++l) {
+        if (pl.write_slot[l] >= 0 && pl.write_before[l])
+            if (int rc = launch_prefill_write(c, pl.write_slot[l], k_layers[l], v_layers[l], n_max, batch, st))
+                return rc;
+        if (int rc = launch_prefill_attention(c, pl.read_slot[l], pl.mode[l], q_layers[l],
+                                              out_layers[l], n_max, batch, st))
+            return rc;
+    }
+    for (int l = 0; l < L; ++l)
+        if (pl.write_slot[l] >= 0 && !pl.write_before[l])
+            if (int rc = launch_prefill_write(c, pl.write_slot[l], k_layers[l], v_layers[l], n_max, batch, st))
+                return rc;
     return LCKV_OK;
 }
 
