@@ -393,6 +393,49 @@ def run_ours(args):
         dist.destroy_process_group()
 
 
+def run_prefill(args):
+    """--prefill N: times the prompt-encoding attention (one layer, condensed mode, N prompt tokens
+    per sequence) and reports tensor-core throughput.  Not the headline metric: a side measurement."""
+    from paper_2405_10637_b200 import binding as lk
+    wl, p = workload_params(args)
+    n = args.prefill
+    B = args.batch or 8
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    cfg = lk.make_config(2, 0, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, B, n)
+    cache = lk.Cache(cfg, device=dev)
+    kt, vt = cache.slot_tensors(0)
+    syn.fill_randn_bf16_(kt, 1, std=wl.std); syn.fill_randn_bf16_(vt, 2, std=wl.std)
+    cache.lckv_cache_reset([n] * B)
+    q = syn.randn_bf16((B, n, wl.n_q_heads, wl.head_dim), 3, device=dev, std=wl.std)
+    out = torch.empty_like(q)
+    stream = torch.cuda.current_stream()
+
+    def f():
+        cache.lckv_prefill_attention(0, lk.MODE_CONDENSED, q, out=out)
+    for _ in range(max(3, args.warmup)):
+        f()
+    torch.cuda.synchronize()
+    ms = time_steps(f, args.steps, stream) / args.steps
+    # visible (i, j) pairs with j < i: n(n-1)/2 per (sequence, head); 4*d flops per pair (QK^T and PV)
+    flops = 4.0 * wl.head_dim * wl.n_q_heads * B * (n * (n - 1) / 2)
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            peak, kind = float(json.load(fh)["bf16_tflops"]), "measured"
+    except Exception:
+        peak, kind = 1590.0, "fallback"
+    tf = flops / (ms * 1e-3) / 1e12
+    print(json.dumps({
+        "metric": "prompt-encoding attention TFLOP/s (causal, useful flops only)", "value": tf,
+        "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": ms, "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{wl.name} head layout, prompt {n}, B={B}, one layer, j<i mask"},
+        "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s",
+                     "frac": tf / peak, "traffic": None, "peak_kind": kind,
+                     "kernel": "prefill_attn_kernel"}}))
+    cache.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -409,6 +452,8 @@ def main():
                     help="s > 0: sink + recent-window caches with s sink tokens, cache size = context")
     ap.add_argument("--ref-rows", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--prefill", type=int, default=0,
+                    help="N > 0: time the prompt-encoding attention on N-token prompts instead")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -416,7 +461,10 @@ def main():
     else:
         if not torch.cuda.is_available():
             raise SystemExit("bench.py needs a CUDA device (the CUDA library has no CPU fallback)")
-        run_ours(args)
+        if args.prefill:
+            run_prefill(args)
+        else:
+            run_ours(args)
 
 
 if __name__ == "__main__":
