@@ -12,6 +12,7 @@
 #include "lckv_attn_alu.cuh"
 #include "lckv_attn_mma.cuh"
 #include "lckv_prefill.cuh"
+#include "lckv_prefill_tc5.cuh"
 #include "lckv_small_kernels.cuh"
 
 namespace {
@@ -91,6 +92,7 @@ struct lckv_cache {
     int n_kv_layers;
     std::vector<CUtensorMap> tm_k, tm_v;  // per slot, tensor-core kernel only
     std::vector<CUtensorMap> tm_pf_k, tm_pf_v;  // per slot, 64-row boxes for prompt encoding
+    int prefill_tc5;                      // 1: prompt encoding on tcgen05, 0: mma.sync kernel
     double l2_keep_bytes;                 // how much of a re-read slot to hold in L2 (0 = off)
     int ws_parity;                        // which half of the split-K workspace the next launch uses
     size_t partials_half_floats;          // floats in one half of the partial records
@@ -144,7 +146,17 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
 
 // Tensor map of one K or V tensor seen as [rows = B_max*H_kv*T_cap, d_h] bf16, box = 64 columns x
 // `box_rows` rows, 128-byte swizzle, out-of-range rows read as zero.
+int make_tensor_map_pitch(CUtensorMap* tm, void* base, uint64_t rows, uint64_t cols,
+                          uint64_t pitch_bytes, int box_rows);
+
 int make_tensor_map(CUtensorMap* tm, void* base, uint64_t rows, int d, int box_rows)
+{
+    return make_tensor_map_pitch(tm, base, rows, (uint64_t)d, (uint64_t)d * 2, box_rows);
+}
+
+// General form: a bf16 matrix of `rows` x `cols` with a row pitch in bytes (multiple of 16).
+int make_tensor_map_pitch(CUtensorMap* tm, void* base, uint64_t rows, uint64_t cols,
+                          uint64_t pitch_bytes, int box_rows)
 {
     static EncodeTiledFn fn = nullptr;
     if (!fn) {
@@ -155,8 +167,8 @@ int make_tensor_map(CUtensorMap* tm, void* base, uint64_t rows, int d, int box_r
         if (q != cudaDriverEntryPointSuccess || !f) return LCKV_ECUDA;
         fn = reinterpret_cast<EncodeTiledFn>(f);
     }
-    const cuuint64_t gdim[2] = {(cuuint64_t)d, (cuuint64_t)rows};
-    const cuuint64_t gstride[1] = {(cuuint64_t)d * 2};
+    const cuuint64_t gdim[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+    const cuuint64_t gstride[1] = {(cuuint64_t)pitch_bytes};
     const cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
     const cuuint32_t estr[2] = {1, 1};
     const CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, base, gdim, gstride, box, estr,
@@ -476,6 +488,25 @@ int launch_prefill_attention(lckv_cache* c, int slot, int mode, const void* q, v
     int longest = 0;
     for (int b = 0; b < batch; ++b) longest = c->h_lens[b] > longest ? c->h_lens[b] : longest;
     if (longest == 0) return LCKV_OK;
+    if (c->prefill_tc5) {
+        // tcgen05 kernel: 128-row query blocks; the Q tile comes through a tensor map built for this
+        // call's q pointer: q seen as [batch * n_max rows, H_q * d_h columns]
+        const uint64_t q_rows = (uint64_t)batch * n_max;
+        if (q_rows >= (1ull << 31)) return LCKV_EINVAL;
+        CUtensorMap tmq;
+        if (int rc = make_tensor_map_pitch(&tmq, const_cast<void*>(q), q_rows,
+                                           (uint64_t)c->cfg.n_q_heads * c->cfg.head_dim,
+                                           (uint64_t)c->cfg.n_q_heads * c->cfg.head_dim * 2, lckv::kT5BM))
+            return rc;
+        const dim3 grid5((longest + lckv::kT5BM - 1) / lckv::kT5BM, c->cfg.n_q_heads, batch);
+        if (c->cfg.head_dim == 128)
+            lckv::prefill_tc5_kernel<128><<<grid5, lckv::kT5Threads, lckv::tc5_smem_bytes<128>(), st>>>(
+                p, tmq, c->tm_pf_k[slot], c->tm_pf_v[slot]);
+        else
+            lckv::prefill_tc5_kernel<64><<<grid5, lckv::kT5Threads, lckv::tc5_smem_bytes<64>(), st>>>(
+                p, tmq, c->tm_pf_k[slot], c->tm_pf_v[slot]);
+        return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
+    }
     const dim3 grid((longest + lckv::kPfBM - 1) / lckv::kPfBM, c->cfg.n_q_heads, batch);
     if (c->cfg.head_dim == 128)
         lckv::prefill_attn_kernel<128><<<grid, lckv::kPfWarps * 32, lckv::prefill_smem_bytes<128>(), st>>>(
@@ -564,6 +595,10 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
         const char* env = getenv("LCKV_L2_KEEP_MB");
         c->l2_keep_bytes = env ? atof(env) * 1e6 : 0.52 * (double)l2;
     }
+    {
+        const char* env = getenv("LCKV_PREFILL_KERNEL");   // "mma" selects the mma.sync kernel
+        c->prefill_tc5 = !(env && env[0] == 'm');
+    }
     c->ws_parity = 0;
     c->partials_half_floats = 2 * (size_t)c->n_workers * partial_record_floats(*cfg);
     c->graph_exec = nullptr;
@@ -591,7 +626,13 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
             }
         }
     }
-    bool ok = cuda_ok(cudaFuncSetAttribute(lckv::prefill_attn_kernel<128>,
+    bool ok = cuda_ok(cudaFuncSetAttribute(lckv::prefill_tc5_kernel<128>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           lckv::tc5_smem_bytes<128>())) &&
+              cuda_ok(cudaFuncSetAttribute(lckv::prefill_tc5_kernel<64>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           lckv::tc5_smem_bytes<64>())) &&
+              cuda_ok(cudaFuncSetAttribute(lckv::prefill_attn_kernel<128>,
                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            lckv::prefill_smem_bytes<128>())) &&
               cuda_ok(cudaFuncSetAttribute(lckv::prefill_attn_kernel<64>,
