@@ -345,10 +345,16 @@ def run_ours(args):
                       "frac_of_measured_peak": gbs / peak, "frac_of_8TBs": gbs / NOMINAL_HBM_GBS})
 
     # ---- end to end through the host-buffer entry point ----------------------------------------
-    hq = [t.cpu().pin_memory() for t in q]
-    hkv = [None if t is None else t.cpu().pin_memory() for t in kv]
-    hout = [torch.empty((B, wl.n_q_heads, wl.head_dim), dtype=torch.bfloat16).pin_memory()
-            for _ in range(L)]
+    # one pinned allocation per tensor kind, sliced per layer (equally spaced -> pitched copies)
+    hq_all = torch.stack([t.cpu() for t in q]).pin_memory()
+    hq = [hq_all[l] for l in range(L)]
+    kv_layers = [l for l in range(L) if kv[l] is not None]
+    hkv_all = torch.stack([kv[l].cpu() for l in kv_layers]).pin_memory()
+    hkv = [None] * L
+    for i, l in enumerate(kv_layers):
+        hkv[l] = hkv_all[i]
+    hout_all = torch.empty((L, B, wl.n_q_heads, wl.head_dim), dtype=torch.bfloat16).pin_memory()
+    hout = [hout_all[l] for l in range(L)]
 
     def e2e_step():
         cache.lckv_layer_stack_step_host(hq, hout, hkv, hkv, batch=B)

@@ -222,7 +222,9 @@ int lckv_layer_stack_step(lckv_cache_t* cache, const void* const* q_layers,
  * real overlap): copies every layer's q (and the k,v of layers that have them)
  * host->device into the cache's staging area, runs the step, copies every
  * layer's output device->host.  All on `stream`, asynchronous; synchronise the
- * stream before reading the outputs.  Needs host_staging = 1 at alloc.
+ * stream before reading the outputs.  Needs host_staging = 1 at alloc.  When the
+ * layers' host buffers are contiguous in memory (one allocation sliced per
+ * layer) each direction is a single pitched copy instead of one copy per layer.
  * Array arguments are HOST arrays of L HOST pointers with the shapes above.
  */
 int lckv_layer_stack_step_host(lckv_cache_t* cache, const void* const* q_layers_host,

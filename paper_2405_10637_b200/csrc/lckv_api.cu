@@ -517,6 +517,36 @@ int launch_prefill_attention(lckv_cache* c, int slot, int mode, const void* q, v
     return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
 }
 
+// Copies `n` equally sized layer buffers between host and the staging area (device pitch
+// `dev_pitch`).  When the host buffers are contiguous (one allocation sliced per layer) this is a
+// single pitched copy; otherwise, or if that copy is refused, one copy per layer.
+int copy_layers(uint8_t* dev, size_t dev_pitch, const void* const* host, int n, size_t bytes,
+                bool to_device, cudaStream_t st)
+{
+    if (n <= 0 || bytes == 0) return LCKV_OK;
+    bool contiguous = n >= 2;
+    for (int l = 1; l < n && contiguous; ++l)
+        contiguous = static_cast<const uint8_t*>(host[l]) ==
+                     static_cast<const uint8_t*>(host[l - 1]) + bytes;
+    if (contiguous) {
+        const cudaError_t e =
+            to_device ? cudaMemcpy2DAsync(dev, dev_pitch, host[0], bytes, bytes, n,
+                                          cudaMemcpyHostToDevice, st)
+                      : cudaMemcpy2DAsync(const_cast<void*>(host[0]), bytes, dev, dev_pitch, bytes, n,
+                                          cudaMemcpyDeviceToHost, st);
+        if (e == cudaSuccess) return LCKV_OK;
+        (void)cudaGetLastError();  // fall back to per-layer copies
+    }
+    for (int l = 0; l < n; ++l) {
+        const cudaError_t e =
+            to_device ? cudaMemcpyAsync(dev + (size_t)l * dev_pitch, host[l], bytes, cudaMemcpyHostToDevice, st)
+                      : cudaMemcpyAsync(const_cast<void*>(host[l]), dev + (size_t)l * dev_pitch, bytes,
+                                        cudaMemcpyDeviceToHost, st);
+        if (!cuda_ok(e)) return LCKV_ECUDA;
+    }
+    return LCKV_OK;
+}
+
 }  // namespace
 
 extern "C" {
@@ -792,29 +822,31 @@ int lckv_layer_stack_step_host(lckv_cache_t* c, const void* const* q_host, void*
     const size_t kv_bytes = (size_t)batch * c->cfg.n_kv_heads * c->cfg.head_dim * 2;
     std::vector<const void*> dq(L), dk(L, nullptr), dv(L, nullptr);
     std::vector<void*> dout(L);
+    std::vector<const void*> hk, hv;
     int kv_i = 0;
     for (int l = 0; l < L; ++l) {
-        uint8_t* sq = c->base + c->lay.off_stage_q + (size_t)l * c->lay.stage_q_bytes;
-        if (!cuda_ok(cudaMemcpyAsync(sq, q_host[l], q_bytes, cudaMemcpyHostToDevice, st)))
-            return LCKV_ECUDA;
-        dq[l] = sq;
+        dq[l] = c->base + c->lay.off_stage_q + (size_t)l * c->lay.stage_q_bytes;
         dout[l] = c->base + c->lay.off_stage_out + (size_t)l * c->lay.stage_out_bytes;
         if (c->plan.write_slot[l] >= 0) {
             uint8_t* sk = c->base + c->lay.off_stage_kv + (size_t)(2 * kv_i) * c->lay.stage_kv_bytes;
-            uint8_t* sv = sk + c->lay.stage_kv_bytes;
-            if (!cuda_ok(cudaMemcpyAsync(sk, kn_host[l], kv_bytes, cudaMemcpyHostToDevice, st)) ||
-                !cuda_ok(cudaMemcpyAsync(sv, vn_host[l], kv_bytes, cudaMemcpyHostToDevice, st)))
-                return LCKV_ECUDA;
             dk[l] = sk;
-            dv[l] = sv;
+            dv[l] = sk + c->lay.stage_kv_bytes;
+            hk.push_back(kn_host[l]);
+            hv.push_back(vn_host[l]);
             ++kv_i;
         }
     }
+    uint8_t* skv = c->base + c->lay.off_stage_kv;
+    if (int rc = copy_layers(c->base + c->lay.off_stage_q, c->lay.stage_q_bytes, q_host, L, q_bytes, true, st))
+        return rc;
+    if (int rc = copy_layers(skv, 2 * c->lay.stage_kv_bytes, hk.data(), (int)hk.size(), kv_bytes, true, st))
+        return rc;
+    if (int rc = copy_layers(skv + c->lay.stage_kv_bytes, 2 * c->lay.stage_kv_bytes, hv.data(),
+                             (int)hv.size(), kv_bytes, true, st))
+        return rc;
     if (int rc = run_step(c, dq.data(), dout.data(), dk.data(), dv.data(), batch, st)) return rc;
-    for (int l = 0; l < L; ++l)
-        if (!cuda_ok(cudaMemcpyAsync(out_host[l], dout[l], o_bytes, cudaMemcpyDeviceToHost, st)))
-            return LCKV_ECUDA;
-    return LCKV_OK;
+    return copy_layers(c->base + c->lay.off_stage_out, c->lay.stage_out_bytes,
+                       const_cast<const void* const*>(out_host), L, o_bytes, false, st);
 }
 
 int lckv_prefill_write_kv(lckv_cache_t* c, int32_t slot, const void* k, const void* v,

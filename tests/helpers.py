@@ -79,14 +79,27 @@ class Case:
               if self.plan["write_slot"][l] >= 0 else None for l in range(self.L)]
         return q, kn, vn
 
-    def step(self, check=True, host=False):
+    def step(self, check=True, host=False, contiguous=False):
         q, kn, vn = self.step_inputs()
         odt = torch.float32 if self.cfg.out_dtype else torch.bfloat16
         if host:
-            qd = [t.pin_memory() for t in q]
-            knd = [None if t is None else t.pin_memory() for t in kn]
-            vnd = [None if t is None else t.pin_memory() for t in vn]
-            outs = [torch.empty((self.B, self.Hq, self.d), dtype=odt).pin_memory() for _ in range(self.L)]
+            if contiguous:   # one pinned block per tensor kind, sliced per layer
+                qa = torch.stack(q).pin_memory()
+                qd = [qa[l] for l in range(self.L)]
+                idx = [l for l in range(self.L) if kn[l] is not None]
+                ka = torch.stack([kn[l] for l in idx]).pin_memory()
+                va = torch.stack([vn[l] for l in idx]).pin_memory()
+                knd, vnd = [None] * self.L, [None] * self.L
+                for i, l in enumerate(idx):
+                    knd[l], vnd[l] = ka[i], va[i]
+                oa = torch.empty((self.L, self.B, self.Hq, self.d), dtype=odt).pin_memory()
+                outs = [oa[l] for l in range(self.L)]
+            else:
+                qd = [t.pin_memory() for t in q]
+                knd = [None if t is None else t.pin_memory() for t in kn]
+                vnd = [None if t is None else t.pin_memory() for t in vn]
+                outs = [torch.empty((self.B, self.Hq, self.d), dtype=odt).pin_memory()
+                        for _ in range(self.L)]
             self.cache.lckv_layer_stack_step_host(qd, outs, knd, vnd)
         else:
             dev = self.cache.device

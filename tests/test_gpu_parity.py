@@ -161,6 +161,11 @@ def test_errors_capacity_and_arguments():
 def test_host_buffer_entry_point_matches():
     c = Case(L=4, w=2, Hq=8, Hkv=8, d=128, lens=[5, 100, 33], T_cap=120, seed=61, host_staging=1)
     c.step(host=True); c.step(host=True)
+    c.step(host=True, contiguous=True); c.step(host=True, contiguous=True)   # single pitched copies
+    c.close()
+    # q bytes per layer not a multiple of the staging pitch (256): pitched copy with padding
+    c = Case(L=3, w=2, Hq=3, Hkv=3, d=64, lens=[5, 9, 33], T_cap=40, seed=62, host_staging=1)
+    c.step(host=True, contiguous=True); c.step(host=True)
     c.close()
 
 
