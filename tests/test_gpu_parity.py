@@ -272,3 +272,64 @@ def test_streaming_sink_and_window_cache(shape):
         c.step()
     assert c.lens.tolist() == [8, 38, 43, 44, 45, 46, 108, 5008]
     c.close()
+
+
+# ---- properties that hold at any size ---------------------------------------------------------------
+
+def _attn_case(Hq, Hkv, d, lens, T_cap, out_dtype=1, seed=0, std=1.0):
+    B = len(lens)
+    cfg = lk.make_config(2, 0, Hq, Hkv, d, B, T_cap, out_dtype=out_dtype)
+    cache = lk.Cache(cfg)
+    K = syn.randn_bf16((B, Hkv, T_cap, d), seed + 1, std=std)
+    V = syn.randn_bf16((B, Hkv, T_cap, d), seed + 2, std=std)
+    kt, vt = cache.slot_tensors(0); kt.copy_(K); vt.copy_(V)
+    cache.lckv_cache_reset(lens)
+    q = syn.randn_bf16((B, Hq, d), seed + 3, std=std).to(cache.device)
+    return cache, K, V, q
+
+
+@pytest.mark.parametrize("Hq,Hkv,d", [(8, 8, 128), (16, 2, 64)])
+def test_rows_at_and_beyond_the_new_token_are_never_read(Hq, Hkv, d):
+    """Diagonal mask: poisoning row t (the position of the new token) and everything after it
+    leaves every condensed output bit-identical."""
+    lens = [0, 7, 16, 100, 255]
+    cache, K, V, q = _attn_case(Hq, Hkv, d, lens, 256, out_dtype=0, seed=10)
+    a = cache.lckv_decode_attention(0, lk.MODE_CONDENSED, q).clone()
+    kt, vt = cache.slot_tensors(0)
+    for b, n in enumerate(lens):
+        kt[b, :, n:] = float("nan"); vt[b, :, n:] = float("nan")
+    bb = cache.lckv_decode_attention(0, lk.MODE_CONDENSED, q)
+    torch.cuda.synchronize()
+    assert np.array_equal(syn.bits(a), syn.bits(bb))
+    cache.close()
+
+
+@pytest.mark.parametrize("Hq,Hkv,d", [(8, 8, 128), (16, 2, 64)])
+def test_joint_permutation_of_cached_rows(Hq, Hkv, d):
+    """Attention does not depend on the order of the visible rows (only on the set)."""
+    lens = [33, 200, 999]
+    cache, K, V, q = _attn_case(Hq, Hkv, d, lens, 1000, seed=20, std=0.5)
+    a = cache.lckv_decode_attention(0, lk.MODE_CONDENSED, q).clone()
+    kt, vt = cache.slot_tensors(0)
+    g = torch.Generator().manual_seed(1)
+    for b, n in enumerate(lens):
+        perm = torch.randperm(n, generator=g).to(cache.device)
+        kt[b, :, :n] = kt[b, :, :n][:, perm]
+        vt[b, :, :n] = vt[b, :, :n][:, perm]
+    p2 = cache.lckv_decode_attention(0, lk.MODE_CONDENSED, q)
+    torch.cuda.synchronize()
+    tol = 1e-5 if Hq == Hkv else 2e-3   # the tensor-core kernel rounds P to bf16 per tile
+    assert (a - p2).abs().max().item() < tol
+    cache.close()
+
+
+def test_a_sequence_does_not_depend_on_its_batch_mates():
+    """Sequences are independent: the first two rows of a batch of five equal a batch of two (up to
+    the summation order, which follows the work split)."""
+    lens = [500, 77, 1000, 3, 640]
+    cache, K, V, q = _attn_case(8, 8, 128, lens, 1024, seed=30)
+    a5 = cache.lckv_decode_attention(0, lk.MODE_CONDENSED, q).clone()
+    a2 = cache.lckv_decode_attention(0, lk.MODE_CONDENSED, q[:2].contiguous(), batch=2)
+    torch.cuda.synchronize()
+    assert (a5[:2] - a2).abs().max().item() < 1e-5
+    cache.close()
