@@ -29,6 +29,8 @@ def build(force: bool = False, verbose: bool = False) -> str:
            os.path.join(CSRC, "lckv_api.cu")]
     if verbose:
         cmd[1:1] = ["-Xptxas", "-v"]
+    extra = os.environ.get("LCKV_NVCC_FLAGS", "").split()   # e.g. tuning macros: -DLCKV_ALU_SLOTS=3
+    cmd[1:1] = extra
     subprocess.run(cmd, check=True)
     os.replace(tmp, LIB)
     return LIB

@@ -262,7 +262,8 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
         const int r = q4 * 32 + lane;                  // row within the block
         const int i = mb * kT5BM + r;                  // prompt position of the row
         const uint32_t lane_sel = (uint32_t)(q4 * 32) << 16;
-        float m_used = -INFINITY, l_run = 0.f;
+        float m_used = -INFINITY, l_run = 0.f;     // m_used in raw (unscaled) score units
+        const float inv_scale = 1.0f / p.scale_log2;
         for (int j = 0; j < n_kv && ok; ++j) {
             ok = mbar_wait_bounded(bSf, j & 1, kT5WaitLimit);
             if (!ok) break;
@@ -270,31 +271,42 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
             uint32_t s0[32], s1[32];
             tmem_ld32(tS + lane_sel, s0);
             tmem_ld32(tS + lane_sel + 32, s1);
+            // Raw scores stay unscaled: the (positive) scale is folded into the exponent's FMA.
             const bool need_mask = (j * kT5BN + kT5BN > mb * kT5BM + p.mode);  // tile reaches the diagonal
             float mt = -INFINITY;
+            if (need_mask) {
+                const int lim = i + p.mode - j * kT5BN;   // columns c < lim are visible
 #pragma unroll
-            for (int c = 0; c < 64; ++c) {
-                float v = __uint_as_float(c < 32 ? s0[c] : s1[c - 32]) * p.scale_log2;
-                if (need_mask && !(j * kT5BN + c < i + p.mode)) v = -INFINITY;
-                if (c < 32) s0[c] = __float_as_uint(v); else s1[c - 32] = __float_as_uint(v);
-                mt = fmaxf(mt, v);
+                for (int c = 0; c < 32; ++c) {
+                    if (c >= lim) s0[c] = 0xff800000u;       // -inf
+                    if (c + 32 >= lim) s1[c] = 0xff800000u;
+                }
             }
-            // Keep the reference maximum unless the new one exceeds it by more than 2^8.
+#pragma unroll
+            for (int c = 0; c < 32; c += 2) {
+                mt = fmaxf(mt, fmaxf(__uint_as_float(s0[c]), __uint_as_float(s0[c + 1])));
+                mt = fmaxf(mt, fmaxf(__uint_as_float(s1[c]), __uint_as_float(s1[c + 1])));
+            }
+            // Keep the reference maximum unless the new one exceeds it by more than 2^8 (in the
+            // exponent's base-2 units): probabilities then stay <= 256.
             float alpha = 1.f;
-            const bool grow = (mt > m_used + 8.f) || (m_used == -INFINITY && mt > -INFINITY);
+            const bool grow = (mt > m_used + 8.f * inv_scale) || (m_used == -INFINITY && mt > -INFINITY);
             if (grow) {
-                alpha = ex2(m_used - mt);              // 0 when nothing was seen before
+                alpha = ex2((m_used - mt) * p.scale_log2);   // 0 when nothing was seen before
                 m_used = mt;
                 l_run *= alpha;
             }
-            const float m_sub = (m_used == -INFINITY) ? 0.f : m_used;
+            const float neg_m = (m_used == -INFINITY) ? 0.f : -m_used * p.scale_log2;
             uint32_t pk[32];
 #pragma unroll
-            for (int c = 0; c < 32; ++c) {
-                const float p0 = ex2(__uint_as_float(c < 16 ? s0[2 * c] : s1[2 * c - 32]) - m_sub);
-                const float p1 = ex2(__uint_as_float(c < 16 ? s0[2 * c + 1] : s1[2 * c - 31]) - m_sub);
+            for (int c = 0; c < 16; ++c) {
+                const float p0 = ex2(fmaf(__uint_as_float(s0[2 * c]), p.scale_log2, neg_m));
+                const float p1 = ex2(fmaf(__uint_as_float(s0[2 * c + 1]), p.scale_log2, neg_m));
+                const float p2 = ex2(fmaf(__uint_as_float(s1[2 * c]), p.scale_log2, neg_m));
+                const float p3 = ex2(fmaf(__uint_as_float(s1[2 * c + 1]), p.scale_log2, neg_m));
                 pk[c] = cvt_bf16x2(p0, p1);
-                l_run += bf16lo(pk[c]) + bf16hi(pk[c]);
+                pk[c + 16] = cvt_bf16x2(p2, p3);
+                l_run += (p0 + p1) + (p2 + p3);
             }
             // P and O are still in use by the previous tile's P V until O_full fires
             if (j > 0) {
