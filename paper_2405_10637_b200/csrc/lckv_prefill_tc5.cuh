@@ -5,15 +5,17 @@
 //
 //   warp 0   producer: TMA loads of the Q tile (once) and of the 64-row K and V tiles
 //   warp 1   one thread issues the MMAs:  S[128x64]  = Q K^T      (A, B from shared memory)
-//                                         O[128xD]  += P V        (P from shared memory, V MN-major)
+//                                         O[128xD]  += P V        (P from tensor memory, V MN-major)
 //            accumulators live in tensor memory; completion is signalled by tcgen05.commit
 //   warps 2-5  one thread per query row (= one tensor-memory lane): read the row of S, mask, running
-//            max (thread-local, no shuffles), probabilities -> bf16 -> shared memory (swizzled), row
-//            sum; rescale the O row in tensor memory only when the maximum grew by more than 2^8
-//            (the probabilities then stay below 256, exact enough in bf16 and fp32); epilogue.
+//            max (thread-local, no shuffles), probabilities -> packed bf16 pairs back into tensor
+//            memory (the A operand of the second MMA), row sum; rescale the O row in tensor memory
+//            only when the maximum grew by more than 2^8 (the probabilities then stay <= 256);
+//            epilogue.
 //
-// Two CTAs fit on an SM (80 KB of shared memory and 256 of the 512 tensor-memory columns each at
-// D = 128), so one CTA's softmax overlaps the other's MMAs.  Every wait is bounded.
+// K and V tiles are double-buffered so that their load latency is hidden behind the previous
+// tile.  Two CTAs fit on an SM (97 KB of shared memory and 256 of the 512 tensor-memory columns
+// each at D = 128), so one CTA's softmax overlaps the other's MMAs.  Every wait is bounded.
 #pragma once
 #include <cuda.h>
 
@@ -29,8 +31,8 @@ constexpr uint32_t kT5WaitLimit = 1u << 16;
 template <int D>
 constexpr int tc5_smem_bytes()
 {
-    // Q [128 x D] + K [64 x D] + V [64 x D] + P [128 x 64], bf16; barriers; alignment slack
-    return kT5BM * D * 2 + 2 * kT5BN * D * 2 + kT5BM * kT5BN * 2 + 128 + 1024;
+    // Q [128 x D] + two stages of K [64 x D] and V [64 x D], bf16; barriers; alignment slack
+    return kT5BM * D * 2 + 4 * kT5BN * D * 2 + 256 + 1024;
 }
 
 // ---- tcgen05 wrappers ----------------------------------------------------------------------------
@@ -58,6 +60,17 @@ __device__ __forceinline__ void tc5_mma(uint32_t d_tmem, uint64_t a_desc, uint64
         "setp.ne.b32 p, %4, 0;\n\t"
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(d_tmem), "l"(a_desc), "l"(b_desc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// Same with the A operand in tensor memory (128 lanes = rows, K elements packed two per column).
+__device__ __forceinline__ void tc5_mma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t b_desc,
+                                           uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate)
         : "memory");
 }
 // The mbarrier receives one arrival once all MMAs issued so far by this thread have completed.
@@ -136,8 +149,8 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
     constexpr int NBOX = D / 64;                   // 64-column boxes per tile
     constexpr int QBOX = kT5BM * 128;              // bytes of one Q box
     constexpr int KBOX = kT5BN * 128;              // bytes of one K or V box
-    constexpr int Q_BYTES = kT5BM * D * 2, KV_BYTES = kT5BN * D * 2, P_BYTES = kT5BM * kT5BN * 2;
-    constexpr uint32_t TM_COLS = (kT5BN + D) <= 128 ? 128 : 256;   // S (64) + O (D), power of two
+    constexpr int Q_BYTES = kT5BM * D * 2, KV_BYTES = kT5BN * D * 2;
+    constexpr uint32_t TM_COLS = 256;   // S (64 fp32) + P (32 columns of bf16 pairs) + O (D fp32), power of two
     constexpr uint32_t IDESC_S = tc5_idesc(kT5BM, kT5BN, 0);
     constexpr uint32_t IDESC_O = tc5_idesc(kT5BM, D, 1);
 
@@ -153,10 +166,11 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
 
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
-    const uint32_t sQ = smem0, sK = sQ + Q_BYTES, sV = sK + KV_BYTES, sP = sV + KV_BYTES;
-    const uint32_t bars = sP + P_BYTES;
-    const uint32_t bQ = bars, bKf = bars + 8, bKe = bars + 16, bVf = bars + 24, bVe = bars + 32,
-                   bSf = bars + 40, bPf = bars + 48, bOf = bars + 56, sTaddr = bars + 64;
+    const uint32_t sQ = smem0, sK = sQ + Q_BYTES, sV = sK + 2 * KV_BYTES;   // K, V: two stages each
+    const uint32_t bars = sV + 2 * KV_BYTES;
+    // per-stage barriers are 8 bytes apart: bKf + 8 * stage etc.
+    const uint32_t bQ = bars, bKf = bars + 8, bKe = bars + 24, bVf = bars + 40, bVe = bars + 56,
+                   bSf = bars + 72, bPf = bars + 80, bOf = bars + 88, sTaddr = bars + 96;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     if (n_kv == 0) {
@@ -171,7 +185,11 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
     }
 
     if (tid == 0) {
-        mbar_init(bQ, 1); mbar_init(bKf, 1); mbar_init(bKe, 1); mbar_init(bVf, 1); mbar_init(bVe, 1);
+        mbar_init(bQ, 1);
+        for (int st = 0; st < 2; ++st) {
+            mbar_init(bKf + 8 * st, 1); mbar_init(bKe + 8 * st, 1);
+            mbar_init(bVf + 8 * st, 1); mbar_init(bVe + 8 * st, 1);
+        }
         mbar_init(bSf, 1); mbar_init(bPf, 128); mbar_init(bOf, 1);
         fence_mbar_init();
     }
@@ -181,7 +199,7 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
     tc5_fence_after();
     uint32_t tmem_base;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sTaddr));
-    const uint32_t tS = tmem_base, tO = tmem_base + kT5BN;
+    const uint32_t tS = tmem_base, tP = tmem_base + kT5BN, tO = tmem_base + kT5BN + kT5BN / 2;
 
     bool ok = true;
     if (warp == 0) {
@@ -192,18 +210,22 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
             for (int bx = 0; bx < NBOX; ++bx)
                 tma_load_2d(sQ + bx * QBOX, &tmQ, h * D + bx * 64, b * p.n_max + mb * kT5BM, bQ);
             for (int j = 0; j < n_kv && ok; ++j) {
-                if (j > 0) ok = mbar_wait_bounded(bKe, (j - 1) & 1, kT5WaitLimit);
+                const int st = j & 1;                    // stage; its k-th use has parity k & 1
+                const uint32_t par_prev = ((j >> 1) - 1) & 1;
+                if (j >= 2) ok = mbar_wait_bounded(bKe + 8 * st, par_prev, kT5WaitLimit);
                 if (!ok) break;
-                mbar_expect_tx(bKf, KV_BYTES);
+                mbar_expect_tx(bKf + 8 * st, KV_BYTES);
 #pragma unroll
                 for (int bx = 0; bx < NBOX; ++bx)
-                    tma_load_2d(sK + bx * KBOX, &tmK, bx * 64, (int32_t)(row0 + (int64_t)j * kT5BN), bKf);
-                if (j > 0) ok = mbar_wait_bounded(bVe, (j - 1) & 1, kT5WaitLimit);
+                    tma_load_2d(sK + st * KV_BYTES + bx * KBOX, &tmK, bx * 64,
+                                (int32_t)(row0 + (int64_t)j * kT5BN), bKf + 8 * st);
+                if (j >= 2) ok = mbar_wait_bounded(bVe + 8 * st, par_prev, kT5WaitLimit);
                 if (!ok) break;
-                mbar_expect_tx(bVf, KV_BYTES);
+                mbar_expect_tx(bVf + 8 * st, KV_BYTES);
 #pragma unroll
                 for (int bx = 0; bx < NBOX; ++bx)
-                    tma_load_2d(sV + bx * KBOX, &tmV, bx * 64, (int32_t)(row0 + (int64_t)j * kT5BN), bVf);
+                    tma_load_2d(sV + st * KV_BYTES + bx * KBOX, &tmV, bx * 64,
+                                (int32_t)(row0 + (int64_t)j * kT5BN), bVf + 8 * st);
             }
             if (!ok) atomicExch(p.status, kStatusTimeout);
         }
@@ -211,47 +233,46 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             ok = mbar_wait_bounded(bQ, 0, kT5WaitLimit);
+            // O += P_t V_t for tile t (P in tensor memory, V tile in stage t & 1)
+            auto issue_pv = [&](int t) {
+                const uint32_t vb = sV + (t & 1) * KV_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < kT5BN / 16; ++ks) {
+                    const uint64_t bd = tc5_desc(vb + ks * 16 * 128, KBOX, 1024);
+                    tc5_mma_ts(tO, tP + ks * 8, bd, IDESC_O, (t > 0 || ks > 0));
+                }
+                tc5_commit(bOf);                 // O (and P) free for the softmax threads
+                tc5_commit(bVe + 8 * (t & 1));   // V stage may be refilled
+            };
             for (int j = 0; j < n_kv && ok; ++j) {
                 // S_j = Q K_j^T : needs K_j, and S free (the rows of S_{j-1} were read: P_{j-1} full)
-                ok = mbar_wait_bounded(bKf, j & 1, kT5WaitLimit);
+                ok = mbar_wait_bounded(bKf + 8 * (j & 1), (j >> 1) & 1, kT5WaitLimit);
                 if (ok && j > 0) ok = mbar_wait_bounded(bPf, (j - 1) & 1, kT5WaitLimit);
                 if (!ok) break;
                 tc5_fence_after();
+                const uint32_t kb = sK + (j & 1) * KV_BYTES;
 #pragma unroll
                 for (int ks = 0; ks < D / 16; ++ks) {
                     const uint64_t ad = tc5_desc(sQ + (ks >> 2) * QBOX + (ks & 3) * 32, 16, 1024);
-                    const uint64_t bd = tc5_desc(sK + (ks >> 2) * KBOX + (ks & 3) * 32, 16, 1024);
+                    const uint64_t bd = tc5_desc(kb + (ks >> 2) * KBOX + (ks & 3) * 32, 16, 1024);
                     tc5_mma(tS, ad, bd, IDESC_S, ks > 0);
                 }
-                tc5_commit(bSf);   // S_j ready for the softmax threads
-                tc5_commit(bKe);   // K buffer may be refilled
+                tc5_commit(bSf);                 // S_j ready for the softmax threads
+                tc5_commit(bKe + 8 * (j & 1));   // K stage may be refilled
                 if (j > 0) {
-                    // O += P_{j-1} V_{j-1}
-                    ok = mbar_wait_bounded(bVf, (j - 1) & 1, kT5WaitLimit);
+                    ok = mbar_wait_bounded(bVf + 8 * ((j - 1) & 1), ((j - 1) >> 1) & 1, kT5WaitLimit);
                     if (!ok) break;
                     tc5_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < kT5BN / 16; ++ks) {
-                        const uint64_t ad = tc5_desc(sP + ks * 32, 16, 1024);
-                        const uint64_t bd = tc5_desc(sV + ks * 16 * 128, KBOX, 1024);
-                        tc5_mma(tO, ad, bd, IDESC_O, (j > 1 || ks > 0));
-                    }
-                    tc5_commit(bOf);
-                    tc5_commit(bVe);
+                    issue_pv(j - 1);
                 }
             }
             if (ok) {
                 const int j = n_kv - 1;  // the last tile's P V
-                ok = mbar_wait_bounded(bPf, j & 1, kT5WaitLimit) && mbar_wait_bounded(bVf, j & 1, kT5WaitLimit);
+                ok = mbar_wait_bounded(bPf, j & 1, kT5WaitLimit) &&
+                     mbar_wait_bounded(bVf + 8 * (j & 1), (j >> 1) & 1, kT5WaitLimit);
                 if (ok) {
                     tc5_fence_after();
-#pragma unroll
-                    for (int ks = 0; ks < kT5BN / 16; ++ks) {
-                        const uint64_t ad = tc5_desc(sP + ks * 32, 16, 1024);
-                        const uint64_t bd = tc5_desc(sV + ks * 16 * 128, KBOX, 1024);
-                        tc5_mma(tO, ad, bd, IDESC_O, (j > 0 || ks > 0));
-                    }
-                    tc5_commit(bOf);
+                    issue_pv(j);
                 }
             }
             if (!ok) atomicExch(p.status, kStatusTimeout);
@@ -324,23 +345,21 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
                     }
                 }
             }
-            // row r of P: 64 bf16 = 8 chunks of 16 bytes, 128-byte swizzle
-#pragma unroll
-            for (int c = 0; c < 8; ++c)
-                sts128(sP + r * 128 + ((c ^ (r & 7)) << 4),
-                       make_uint4(pk[4 * c], pk[4 * c + 1], pk[4 * c + 2], pk[4 * c + 3]));
+            // row r of P: 64 bf16 as 32 packed pairs = 32 tensor-memory columns of this lane
+            tmem_st32(tP + lane_sel, pk);
             if (j * kT5BN + kT5BN > nb) {
                 // rows of V past the prompt came with the box: weight 0, but 0 * NaN = NaN
-                ok = mbar_wait_bounded(bVf, j & 1, kT5WaitLimit);
+                ok = mbar_wait_bounded(bVf + 8 * (j & 1), (j >> 1) & 1, kT5WaitLimit);
                 if (!ok) break;
                 const int first = nb - j * kT5BN;
                 const int t128 = tid - 64;
+                const uint32_t vb = sV + (j & 1) * KV_BYTES;
 #pragma unroll
                 for (int bx = 0; bx < NBOX; ++bx)
                     for (int x = first * 128 + t128 * 16; x < KBOX; x += 128 * 16)
-                        sts128(sV + bx * KBOX + x, make_uint4(0, 0, 0, 0));
+                        sts128(vb + bx * KBOX + x, make_uint4(0, 0, 0, 0));
+                fence_proxy_async_smem();   // generic writes -> visible to the MMA's reads
             }
-            fence_proxy_async_smem();   // generic writes (P, zeroed V rows) -> visible to the MMA
             tc5_fence_before();
             mbar_arrive(bPf);
         }
