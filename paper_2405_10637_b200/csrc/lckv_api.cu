@@ -126,7 +126,9 @@ int validate_config(const lckv_config_t* c)
 int resolve_kernel_kind(const lckv_config_t& c)
 {
     const int g = c.n_q_heads / c.n_kv_heads;
-    return (c.kernel_kind == 0 && g % 8 == 0) ? 2 : 1;
+    // the tensor-core kernel addresses cache rows through 32-bit TMA coordinates
+    const uint64_t rows = (uint64_t)c.max_batch * c.n_kv_heads * (uint64_t)c.max_seq;
+    return (c.kernel_kind == 0 && g % 8 == 0 && rows < (1ull << 31)) ? 2 : 1;
 }
 
 int workers_per_sm(const lckv_config_t& c)

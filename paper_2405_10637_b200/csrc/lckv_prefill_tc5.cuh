@@ -100,6 +100,21 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t (&r)[32])
         : "memory");
     asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
 }
+__device__ __forceinline__ void tmem_ld32_nowait(uint32_t taddr, uint32_t (&r)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,"
+        "%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]),
+          "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]),
+          "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]),
+          "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 __device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t (&r)[32])
 {
     asm volatile(
@@ -150,7 +165,7 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
     constexpr int QBOX = kT5BM * 128;              // bytes of one Q box
     constexpr int KBOX = kT5BN * 128;              // bytes of one K or V box
     constexpr int Q_BYTES = kT5BM * D * 2, KV_BYTES = kT5BN * D * 2;
-    constexpr uint32_t TM_COLS = 256;   // S (64 fp32) + P (32 columns of bf16 pairs) + O (D fp32), power of two
+    constexpr uint32_t TM_COLS = 256;   // 2 x S/P (64 columns each) + O (D fp32), power of two
     constexpr uint32_t IDESC_S = tc5_idesc(kT5BM, kT5BN, 0);
     constexpr uint32_t IDESC_O = tc5_idesc(kT5BM, D, 1);
 
@@ -170,7 +185,7 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
     const uint32_t bars = sV + 2 * KV_BYTES;
     // per-stage barriers are 8 bytes apart: bKf + 8 * stage etc.
     const uint32_t bQ = bars, bKf = bars + 8, bKe = bars + 24, bVf = bars + 40, bVe = bars + 56,
-                   bSf = bars + 72, bPf = bars + 80, bOf = bars + 88, sTaddr = bars + 96;
+                   bSf = bars + 72, bPf = bars + 88, bOf = bars + 96, sTaddr = bars + 104;
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
 
     if (n_kv == 0) {
@@ -190,7 +205,7 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
             mbar_init(bKf + 8 * st, 1); mbar_init(bKe + 8 * st, 1);
             mbar_init(bVf + 8 * st, 1); mbar_init(bVe + 8 * st, 1);
         }
-        mbar_init(bSf, 1); mbar_init(bPf, 128); mbar_init(bOf, 1);
+        mbar_init(bSf, 1); mbar_init(bSf + 8, 1); mbar_init(bPf, 128); mbar_init(bOf, 1);
         fence_mbar_init();
     }
     if (warp == 0) tmem_alloc(sTaddr, TM_COLS);
@@ -199,7 +214,9 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
     tc5_fence_after();
     uint32_t tmem_base;
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sTaddr));
-    const uint32_t tS = tmem_base, tP = tmem_base + kT5BN, tO = tmem_base + kT5BN + kT5BN / 2;
+    // Tensor memory: two score buffers of 64 columns (tile j uses buffer j & 1; the bf16 pairs of
+    // P_j overwrite the first 32 columns of S_j once the row has been read), then O.
+    const uint32_t tSP = tmem_base, tO = tmem_base + 2 * kT5BN;
 
     bool ok = true;
     if (warp == 0) {
@@ -233,47 +250,46 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
         // ------------------------------------------------------------------ MMA issuer
         if (lane == 0) {
             ok = mbar_wait_bounded(bQ, 0, kT5WaitLimit);
-            // O += P_t V_t for tile t (P in tensor memory, V tile in stage t & 1)
+            // S_t = Q K_t^T into score buffer t & 1
+            auto issue_s = [&](int t) {
+                const uint32_t kb = sK + (t & 1) * KV_BYTES;
+#pragma unroll
+                for (int ks = 0; ks < D / 16; ++ks) {
+                    const uint64_t ad = tc5_desc(sQ + (ks >> 2) * QBOX + (ks & 3) * 32, 16, 1024);
+                    const uint64_t bd = tc5_desc(kb + (ks >> 2) * KBOX + (ks & 3) * 32, 16, 1024);
+                    tc5_mma(tSP + (t & 1) * kT5BN, ad, bd, IDESC_S, ks > 0);
+                }
+                tc5_commit(bSf + 8 * (t & 1));   // S_t ready for the softmax threads
+                tc5_commit(bKe + 8 * (t & 1));   // K stage may be refilled
+            };
+            // O += P_t V_t (P in tensor memory, buffer t & 1; V tile in stage t & 1)
             auto issue_pv = [&](int t) {
                 const uint32_t vb = sV + (t & 1) * KV_BYTES;
 #pragma unroll
                 for (int ks = 0; ks < kT5BN / 16; ++ks) {
                     const uint64_t bd = tc5_desc(vb + ks * 16 * 128, KBOX, 1024);
-                    tc5_mma_ts(tO, tP + ks * 8, bd, IDESC_O, (t > 0 || ks > 0));
+                    tc5_mma_ts(tO, tSP + (t & 1) * kT5BN + ks * 8, bd, IDESC_O, (t > 0 || ks > 0));
                 }
-                tc5_commit(bOf);                 // O (and P) free for the softmax threads
+                tc5_commit(bOf);                 // O free for rescaling, score buffer t & 1 reusable
                 tc5_commit(bVe + 8 * (t & 1));   // V stage may be refilled
             };
+            if (ok) ok = mbar_wait_bounded(bKf, 0, kT5WaitLimit);
+            if (ok) { tc5_fence_after(); issue_s(0); }
             for (int j = 0; j < n_kv && ok; ++j) {
-                // S_j = Q K_j^T : needs K_j, and S free (the rows of S_{j-1} were read: P_{j-1} full)
-                ok = mbar_wait_bounded(bKf + 8 * (j & 1), (j >> 1) & 1, kT5WaitLimit);
-                if (ok && j > 0) ok = mbar_wait_bounded(bPf, (j - 1) & 1, kT5WaitLimit);
-                if (!ok) break;
-                tc5_fence_after();
-                const uint32_t kb = sK + (j & 1) * KV_BYTES;
-#pragma unroll
-                for (int ks = 0; ks < D / 16; ++ks) {
-                    const uint64_t ad = tc5_desc(sQ + (ks >> 2) * QBOX + (ks & 3) * 32, 16, 1024);
-                    const uint64_t bd = tc5_desc(kb + (ks >> 2) * KBOX + (ks & 3) * 32, 16, 1024);
-                    tc5_mma(tS, ad, bd, IDESC_S, ks > 0);
-                }
-                tc5_commit(bSf);                 // S_j ready for the softmax threads
-                tc5_commit(bKe + 8 * (j & 1));   // K stage may be refilled
-                if (j > 0) {
-                    ok = mbar_wait_bounded(bVf + 8 * ((j - 1) & 1), ((j - 1) >> 1) & 1, kT5WaitLimit);
+                if (j + 1 < n_kv) {
+                    // scores of the next tile, one tile ahead of the softmax: needs K_{j+1} and the
+                    // buffer (j+1) & 1, whose last user was P_{j-1} V_{j-1}
+                    ok = mbar_wait_bounded(bKf + 8 * ((j + 1) & 1), ((j + 1) >> 1) & 1, kT5WaitLimit);
+                    if (ok && j >= 1) ok = mbar_wait_bounded(bOf, (j - 1) & 1, kT5WaitLimit);
                     if (!ok) break;
                     tc5_fence_after();
-                    issue_pv(j - 1);
+                    issue_s(j + 1);
                 }
-            }
-            if (ok) {
-                const int j = n_kv - 1;  // the last tile's P V
                 ok = mbar_wait_bounded(bPf, j & 1, kT5WaitLimit) &&
                      mbar_wait_bounded(bVf + 8 * (j & 1), (j >> 1) & 1, kT5WaitLimit);
-                if (ok) {
-                    tc5_fence_after();
-                    issue_pv(j);
-                }
+                if (!ok) break;
+                tc5_fence_after();
+                issue_pv(j);
             }
             if (!ok) atomicExch(p.status, kStatusTimeout);
         }
@@ -286,12 +302,14 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
         float m_used = -INFINITY, l_run = 0.f;     // m_used in raw (unscaled) score units
         const float inv_scale = 1.0f / p.scale_log2;
         for (int j = 0; j < n_kv && ok; ++j) {
-            ok = mbar_wait_bounded(bSf, j & 1, kT5WaitLimit);
+            ok = mbar_wait_bounded(bSf + 8 * (j & 1), (j >> 1) & 1, kT5WaitLimit);
             if (!ok) break;
             tc5_fence_after();
             uint32_t s0[32], s1[32];
-            tmem_ld32(tS + lane_sel, s0);
-            tmem_ld32(tS + lane_sel + 32, s1);
+            const uint32_t tbuf = tSP + (j & 1) * kT5BN + lane_sel;
+            tmem_ld32_nowait(tbuf, s0);
+            tmem_ld32_nowait(tbuf + 32, s1);
+            tmem_ld_wait();
             // Raw scores stay unscaled: the (positive) scale is folded into the exponent's FMA.
             const bool need_mask = (j * kT5BN + kT5BN > mb * kT5BM + p.mode);  // tile reaches the diagonal
             float mt = -INFINITY;
@@ -346,7 +364,7 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
                 }
             }
             // row r of P: 64 bf16 as 32 packed pairs = 32 tensor-memory columns of this lane
-            tmem_st32(tP + lane_sel, pk);
+            tmem_st32(tbuf, pk);
             if (j * kT5BN + kT5BN > nb) {
                 // rows of V past the prompt came with the box: weight 0, but 0 * NaN = NaN
                 ok = mbar_wait_bounded(bVf + 8 * (j & 1), (j >> 1) & 1, kT5WaitLimit);
