@@ -245,15 +245,20 @@ def run_ours(args):
     wl, p = workload_params(args)
     B, T_cap = p["batch"], p["t_cap"]
     L = wl.n_layers
+    # every rank draws its own sequences (different seeds): independent replicas of the workload
+    lens = syn.ragged_lengths(B, p["lo"], p["hi"], syn.seed_for(wl, syn.T_LENS, rank)).numpy()
+    n_pages = 0
+    if args.page_rows:   # pool: what the sequences hold at the end of the longest timed run, + 2 %
+        grow = max(64, args.steps + args.warmup + 8)
+        n_pages = int(1.02 * sum((int(x) + grow + args.page_rows - 1) // args.page_rows for x in lens)) + 8
     cfg = lk.make_config(L, wl.n_warmup, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, B, T_cap,
                          host_staging=1, use_graph=1 if args.graph else 0,
-                         top_variant=args.top_variant, stream_sink=args.stream_sink)
+                         top_variant=args.top_variant, stream_sink=args.stream_sink,
+                         page_rows=args.page_rows, n_pages=n_pages)
     cap = T_cap if args.stream_sink else 0
     cache = lk.Cache(cfg, device=dev)
     plan = lk.lckv_plan(L, wl.n_warmup, args.top_variant)
     info = cache.info
-    # every rank draws its own sequences (different seeds): independent replicas of the workload
-    lens = syn.ragged_lengths(B, p["lo"], p["hi"], syn.seed_for(wl, syn.T_LENS, rank)).numpy()
     for s in range(info.n_slots):
         kt, vt = cache.slot_tensors(s)
         syn.fill_randn_bf16_(kt, syn.seed_for(wl, syn.T_K, s + 16 * rank), std=wl.std)
@@ -368,7 +373,7 @@ def run_ours(args):
 
     # ---- CPU baseline: the checker on a bounded sample (rank 0, N = 1 only) --------------------
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline and not args.stream_sink:
+    if rank == 0 and world == 1 and not (args.no_cpu_baseline or args.stream_sink or args.page_rows):
         rows = min(args.ref_rows, B)
         Ks = [syn.bits(cache.slot_tensors(s)[0][:rows]) for s in range(info.n_slots)]
         Vs = [syn.bits(cache.slot_tensors(s)[1][:rows]) for s in range(info.n_slots)]
@@ -388,7 +393,8 @@ def run_ours(args):
                        if 2 * info.slot_bytes > 2 * 126e6 else "L2-resident cache: warm",
                        "kv_bytes_per_step": bytes_step, "footprint_slots": info.n_slots,
                        "top_variant": args.top_variant, "graph": bool(args.graph),
-                       "stream_sink": args.stream_sink},
+                       "stream_sink": args.stream_sink, "page_rows": args.page_rows,
+                       "cache_bytes": int(2 * info.n_slots * info.slot_bytes)},
             "frac_of_8TBs": value / world / NOMINAL_HBM_GBS,
             "clocks": clocks, "e2e": e2e, "gpu_launches": info.launches_per_step * args.steps,
             "roofline": roofline, "cpu_baseline": cpu, "sweep": sweep,
@@ -454,6 +460,8 @@ def main():
     ap.add_argument("--warmup-layers", type=int, default=None, help="override w")
     ap.add_argument("--top-variant", type=int, default=0)
     ap.add_argument("--graph", type=int, default=1)
+    ap.add_argument("--page-rows", type=int, default=0,
+                    help="P > 0: paged caches with P-row pages and a pool sized for the batch's lengths")
     ap.add_argument("--stream-sink", type=int, default=0,
                     help="s > 0: sink + recent-window caches with s sink tokens, cache size = context")
     ap.add_argument("--ref-rows", type=int, default=32)

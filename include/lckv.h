@@ -76,6 +76,13 @@ typedef struct {
                               recent max_seq - s tokens; token t >= max_seq overwrites row
                               s + (t - s) mod (max_seq - s).  Lengths keep counting all tokens;
                               LCKV_ECAPACITY is never returned.  Needs 1 <= s < max_seq.     */
+    int32_t page_rows;     /* 0 = each slot is one [B_max, H_kv, T_cap, d_h] tensor.  P > 0 (a power of
+                              two >= 64): paged slots [n_pages, H_kv, P, d_h]; a sequence owns
+                              ceil(len / P) pages taken from a pool, so ragged batches pay for the
+                              rows they hold, not for B_max * T_cap.  One page table
+                              [B_max][ceil(T_cap / P)] serves every slot (all caches have the same
+                              lengths).  Not combinable with stream_sink.                     */
+    int32_t n_pages;       /* pool size per slot when page_rows > 0                            */
     int32_t kernel_kind;   /* 0 = choose (tensor-core kernel when the query group is a dense
                               MMA tile, else the FP32-ALU kernel); 1 = force FP32-ALU        */
 } lckv_config_t;
@@ -167,6 +174,16 @@ int lckv_cache_status(const lckv_cache_t* cache, int32_t* host_status, void* str
 /* Device pointers of slot `slot`'s K and V tensors [B_max, H_kv, T_cap, d_h] bf16 (for filling
  * a cache with a prompt's keys and values, or inspecting it).  EINVAL on bad slot / null. */
 int lckv_cache_slot_ptrs(const lckv_cache_t* cache, int32_t slot, void** k, void** v);
+
+/*
+ * Paged caches only: copies the host mirror of the page table, [max_batch][*entries_per_seq] page
+ * ids (-1 = no page), to host_out (may be NULL to query the width only).  Logical row r of
+ * sequence b is row r % page_rows of page table[b][r / page_rows], i.e. element
+ * [page, kv_head, r % page_rows, :] of a slot tensor.  Pages are assigned by lckv_cache_reset and,
+ * as sequences grow, by the append / step calls; when the pool is exhausted those calls return
+ * LCKV_ECAPACITY and change nothing.  EINVAL if the cache is not paged.
+ */
+int lckv_cache_page_table(const lckv_cache_t* cache, int32_t* host_out, int32_t* entries_per_seq);
 
 /*
  * Append (Section 2.1: only the top layer and the warmup layers compute K/V):

@@ -20,7 +20,8 @@ class Config(C.Structure):
                 ("n_q_heads", C.c_int32), ("n_kv_heads", C.c_int32), ("head_dim", C.c_int32),
                 ("max_batch", C.c_int32), ("max_seq", C.c_int32), ("softmax_scale", C.c_float),
                 ("top_variant", C.c_int32), ("out_dtype", C.c_int32), ("host_staging", C.c_int32),
-                ("use_graph", C.c_int32), ("stream_sink", C.c_int32), ("kernel_kind", C.c_int32)]
+                ("use_graph", C.c_int32), ("stream_sink", C.c_int32), ("page_rows", C.c_int32), ("n_pages", C.c_int32),
+                ("kernel_kind", C.c_int32)]
 
 
 class Info(C.Structure):
@@ -43,6 +44,7 @@ SIGNATURES = {
     "lckv_cache_lengths": (C.c_int, [_vp, _i32p, _i32, _vp]),
     "lckv_cache_status": (C.c_int, [_vp, _i32p, _vp]),
     "lckv_cache_slot_ptrs": (C.c_int, [_vp, _i32, _vpp, _vpp]),
+    "lckv_cache_page_table": (C.c_int, [_vp, _i32p, _i32p]),
     "lckv_append_kv": (C.c_int, [_vp, _i32, _vp, _vp, _i32, _i32, _vp]),
     "lckv_decode_attention": (C.c_int, [_vp, _i32, _i32, _vp, _vp, _vp, _i32, _vp]),
     "lckv_layer_stack_step": (C.c_int, [_vp, _vpp, _vpp, _vpp, _vpp, _i32, _vp]),
@@ -116,10 +118,10 @@ def lckv_plan(n_layers, n_warmup, top_variant=0):
 
 def make_config(n_layers, n_warmup, n_q_heads, n_kv_heads, head_dim, max_batch, max_seq,
                 softmax_scale=0.0, top_variant=0, out_dtype=0, host_staging=0, use_graph=0,
-                kernel_kind=0, stream_sink=0):
+                kernel_kind=0, stream_sink=0, page_rows=0, n_pages=0):
     return Config(C.sizeof(Config), n_layers, n_warmup, n_q_heads, n_kv_heads, head_dim,
                   max_batch, max_seq, softmax_scale, top_variant, out_dtype, host_staging,
-                  use_graph, stream_sink, kernel_kind)
+                  use_graph, stream_sink, page_rows, n_pages, kernel_kind)
 
 
 def lckv_cache_bytes(cfg):
@@ -201,12 +203,23 @@ class Cache:
              "lckv_cache_slot_ptrs")
         return k.value, v.value
 
+    def lckv_cache_page_table(self):
+        """Paged caches: torch int64 tensor [B_max, entries_per_seq] of page ids (-1 = none)."""
+        n = C.c_int32(0)
+        _chk(lib().lckv_cache_page_table(self.h, None, C.byref(n)), "lckv_cache_page_table")
+        arr = (C.c_int32 * (self.cfg.max_batch * n.value))()
+        _chk(lib().lckv_cache_page_table(self.h, arr, C.byref(n)), "lckv_cache_page_table")
+        return torch.tensor(list(arr), dtype=torch.int64).view(self.cfg.max_batch, n.value)
+
     def slot_tensors(self, slot):
-        """torch views [B_max, H_kv, T_cap, d_h] bf16 of a slot's K and V (same memory)."""
+        """torch views of a slot's K and V (same memory): [B_max, H_kv, T_cap, d_h] bf16, or
+        [n_pages, H_kv, page_rows, d_h] for a paged cache."""
         k, v = self.lckv_cache_slot_ptrs(slot)
         c = self.cfg
         shape = (c.max_batch, c.n_kv_heads, c.max_seq, c.head_dim)
-        n = 2 * c.max_batch * c.n_kv_heads * c.max_seq * c.head_dim
+        if c.page_rows:
+            shape = (c.n_pages, c.n_kv_heads, c.page_rows, c.head_dim)
+        n = 2 * shape[0] * shape[1] * shape[2] * shape[3]
         base = self.buf.data_ptr()
         kt = self.buf[k - base:k - base + n].view(torch.bfloat16).view(shape)
         vt = self.buf[v - base:v - base + n].view(torch.bfloat16).view(shape)

@@ -66,6 +66,7 @@ int make_plan(int L, int w, int variant, Plan& pl)
 }
 
 struct Layout {
+    size_t off_pt;
     size_t off_lens, off_pre, off_start, off_counters, off_status, off_partials, off_slots;
     size_t off_stage_q, off_stage_out, off_stage_kv;
     size_t slot_bytes, workspace_bytes, total_bytes;
@@ -92,6 +93,13 @@ struct lckv_cache {
     int n_kv_layers;
     std::vector<CUtensorMap> tm_k, tm_v;  // per slot, tensor-core kernel only
     std::vector<CUtensorMap> tm_pf_k, tm_pf_v;  // per slot, 64-row boxes for prompt encoding
+    // paged caches (cfg.page_rows > 0): page table mirror and the pool's free list
+    int pt_stride, page_shift;
+    int32_t* d_pt;
+    std::vector<int32_t> h_pt;            // [max_batch][pt_stride], -1 = none
+    std::vector<int32_t> n_pages_of;      // pages held per sequence
+    std::vector<int32_t> free_pages;      // stack of free page ids
+    bool pt_dirty;
     int prefill_tc5;                      // 1: prompt encoding on tcgen05, 0: mma.sync kernel
     double l2_keep_bytes;                 // how much of a re-read slot to hold in L2 (0 = off)
     int ws_parity;                        // which half of the split-K workspace the next launch uses
@@ -114,6 +122,10 @@ int validate_config(const lckv_config_t* c)
     if (c->out_dtype != 0 && c->out_dtype != 1) return LCKV_EINVAL;
     if (c->kernel_kind != 0 && c->kernel_kind != 1) return LCKV_EINVAL;
     if (c->stream_sink < 0 || (c->stream_sink > 0 && c->stream_sink >= c->max_seq)) return LCKV_EINVAL;
+    if (c->page_rows != 0) {
+        const int P = c->page_rows;
+        if (P < 64 || P > 65536 || (P & (P - 1)) || c->n_pages < 1 || c->stream_sink > 0) return LCKV_EINVAL;
+    }
     Plan pl;
     if (int rc = make_plan(c->n_layers, c->n_warmup, c->top_variant, pl)) return rc;
     // tile counts are kept in 32 bits
@@ -127,7 +139,8 @@ int resolve_kernel_kind(const lckv_config_t& c)
 {
     const int g = c.n_q_heads / c.n_kv_heads;
     // the tensor-core kernel addresses cache rows through 32-bit TMA coordinates
-    const uint64_t rows = (uint64_t)c.max_batch * c.n_kv_heads * (uint64_t)c.max_seq;
+    const uint64_t rows = c.page_rows ? (uint64_t)c.n_pages * c.n_kv_heads * (uint64_t)c.page_rows
+                                      : (uint64_t)c.max_batch * c.n_kv_heads * (uint64_t)c.max_seq;
     return (c.kernel_kind == 0 && g % 8 == 0 && rows < (1ull << 31)) ? 2 : 1;
 }
 
@@ -195,9 +208,13 @@ void make_layout(const lckv_config_t& c, int n_slots, int n_workers, int n_kv_la
     y.off_status = off;    off = align_up(off + 4, A);
     y.off_partials = off;
     off = align_up(off + 2 * 2 * (size_t)n_workers * partial_record_floats(c) * 4, A);  // two halves
-    y.workspace_bytes = off;
     y.slot_bytes =
-        align_up((size_t)c.max_batch * c.n_kv_heads * (size_t)c.max_seq * c.head_dim * 2, A);
+        c.page_rows ? align_up((size_t)c.n_pages * c.n_kv_heads * (size_t)c.page_rows * c.head_dim * 2, A)
+                    : align_up((size_t)c.max_batch * c.n_kv_heads * (size_t)c.max_seq * c.head_dim * 2, A);
+    y.off_pt = off;
+    if (c.page_rows)
+        off = align_up(off + (size_t)c.max_batch * ((c.max_seq + c.page_rows - 1) / c.page_rows) * 4, A);
+    y.workspace_bytes = off;
     y.off_slots = off;     off += 2 * (size_t)n_slots * y.slot_bytes;
     y.stage_q_bytes = align_up((size_t)c.max_batch * c.n_q_heads * c.head_dim * 2, A);
     y.stage_out_bytes =
@@ -237,6 +254,77 @@ int max_len(const lckv_cache* c, int batch)
     int m = 0;
     for (int b = 0; b < batch; ++b) m = c->h_lens[b] > m ? c->h_lens[b] : m;
     return m;
+}
+
+// Paged caches: make sure every sequence b < batch owns pages for h_lens[b] + extra rows, taking
+// pages from the pool.  On exhaustion nothing is changed and LCKV_ECAPACITY is returned.
+int ensure_pages(lckv_cache* c, int batch, int extra)
+{
+    if (!c->cfg.page_rows) return LCKV_OK;
+    std::vector<std::pair<int, int>> taken;  // (sequence, page) for roll-back
+    for (int b = 0; b < batch; ++b) {
+        const int rows = c->h_lens[b] + extra;
+        if (rows > c->cfg.max_seq) break;  // reported by the caller's own capacity check
+        const int need = (rows + c->cfg.page_rows - 1) >> c->page_shift;
+        while (c->n_pages_of[b] < need) {
+            if (c->free_pages.empty()) {
+                for (auto it = taken.rbegin(); it != taken.rend(); ++it) {
+                    c->free_pages.push_back(it->second);
+                    c->h_pt[(size_t)it->first * c->pt_stride + --c->n_pages_of[it->first]] = -1;
+                }
+                return LCKV_ECAPACITY;
+            }
+            const int pg = c->free_pages.back();
+            c->free_pages.pop_back();
+            c->h_pt[(size_t)b * c->pt_stride + c->n_pages_of[b]++] = pg;
+            taken.emplace_back(b, pg);
+        }
+    }
+    if (!taken.empty()) c->pt_dirty = true;
+    return LCKV_OK;
+}
+
+// Paged caches, on reset: sequences b < batch give their pages back and get ceil(len / P) new ones.
+// Checked first, so that a pool too small for the request changes nothing.
+int repage(lckv_cache* c, const int32_t* lens, int batch)
+{
+    if (!c->cfg.page_rows) return LCKV_OK;
+    size_t need = 0, held = 0;
+    for (int b = 0; b < batch; ++b) {
+        const int rows = lens ? lens[b] : 0;
+        if (rows > c->cfg.max_seq) return LCKV_ECAPACITY;
+        need += (size_t)((rows + c->cfg.page_rows - 1) >> c->page_shift);
+        held += (size_t)c->n_pages_of[b];
+    }
+    if (need > c->free_pages.size() + held) return LCKV_ECAPACITY;
+    for (int b = 0; b < batch; ++b) {
+        while (c->n_pages_of[b] > 0) {
+            int32_t& e = c->h_pt[(size_t)b * c->pt_stride + --c->n_pages_of[b]];
+            c->free_pages.push_back(e);
+            e = -1;
+        }
+    }
+    for (int b = 0; b < batch; ++b) {
+        const int rows = lens ? lens[b] : 0;
+        const int n = (rows + c->cfg.page_rows - 1) >> c->page_shift;
+        for (int i = 0; i < n; ++i) {
+            c->h_pt[(size_t)b * c->pt_stride + i] = c->free_pages.back();
+            c->free_pages.pop_back();
+        }
+        c->n_pages_of[b] = n;
+    }
+    c->pt_dirty = true;
+    return LCKV_OK;
+}
+
+// Upload the page table if it changed since the last upload (pageable source: staged before return).
+int sync_page_table(lckv_cache* c, cudaStream_t st)
+{
+    if (!c->cfg.page_rows || !c->pt_dirty) return LCKV_OK;
+    if (!cuda_ok(cudaMemcpyAsync(c->d_pt, c->h_pt.data(), c->h_pt.size() * 4, cudaMemcpyHostToDevice, st)))
+        return LCKV_ECUDA;
+    c->pt_dirty = false;
+    return LCKV_OK;
 }
 
 int launch_plan(lckv_cache* c, int batch, cudaStream_t st)
@@ -295,6 +383,10 @@ int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out
     p.scale_log2 = c->scale_log2;
     p.early_kv = early ? 1 : 0;
     p.l2_keep = l2_keep;
+    p.page_table = c->d_pt;
+    p.pt_stride = c->pt_stride;
+    p.page_shift = c->page_shift;
+    const bool paged = c->cfg.page_rows != 0;
     cudaError_t e;
     if (c->kernel_kind == 2) {
         lckv::MmaParams mp;
@@ -302,18 +394,23 @@ int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out
         mp.a.H_q = c->h_pairs;  // pairs per sequence = groups of 8 query heads
         mp.n_q_heads = c->cfg.n_q_heads;
         mp.groups_per_kv = c->cfg.n_q_heads / c->cfg.n_kv_heads / 8;
+        const int blk = lckv::kMmaWarps * 32;
+        const size_t sm = lckv::kMmaSmemBytes;
         if (c->cfg.head_dim == 128)
-            e = launch_pdl(lckv::attn_mma_kernel<128>, c->grid, lckv::kMmaWarps * 32,
-                           lckv::kMmaSmemBytes, st, mp, c->tm_k[slot], c->tm_v[slot]);
+            e = paged ? launch_pdl(lckv::attn_mma_kernel<128, true>, c->grid, blk, sm, st, mp, c->tm_k[slot], c->tm_v[slot])
+                      : launch_pdl(lckv::attn_mma_kernel<128, false>, c->grid, blk, sm, st, mp, c->tm_k[slot], c->tm_v[slot]);
         else
-            e = launch_pdl(lckv::attn_mma_kernel<64>, c->grid, lckv::kMmaWarps * 32,
-                           lckv::kMmaSmemBytes, st, mp, c->tm_k[slot], c->tm_v[slot]);
-    } else if (c->cfg.head_dim == 128) {
-        e = launch_pdl(lckv::attn_alu_kernel<128>, c->grid, lckv::kAluWarps * 32,
-                       lckv::kAluSmemBytes, st, p);
+            e = paged ? launch_pdl(lckv::attn_mma_kernel<64, true>, c->grid, blk, sm, st, mp, c->tm_k[slot], c->tm_v[slot])
+                      : launch_pdl(lckv::attn_mma_kernel<64, false>, c->grid, blk, sm, st, mp, c->tm_k[slot], c->tm_v[slot]);
     } else {
-        e = launch_pdl(lckv::attn_alu_kernel<64>, c->grid, lckv::kAluWarps * 32,
-                       lckv::kAluSmemBytes, st, p);
+        const int blk = lckv::kAluWarps * 32;
+        const size_t sm = lckv::kAluSmemBytes;
+        if (c->cfg.head_dim == 128)
+            e = paged ? launch_pdl(lckv::attn_alu_kernel<128, true>, c->grid, blk, sm, st, p)
+                      : launch_pdl(lckv::attn_alu_kernel<128, false>, c->grid, blk, sm, st, p);
+        else
+            e = paged ? launch_pdl(lckv::attn_alu_kernel<64, true>, c->grid, blk, sm, st, p)
+                      : launch_pdl(lckv::attn_alu_kernel<64, false>, c->grid, blk, sm, st, p);
     }
     return cuda_ok(e) ? LCKV_OK : LCKV_ECUDA;
 }
@@ -327,7 +424,7 @@ int launch_append(lckv_cache* c, int slot, const void* k_new, const void* v_new,
     lckv::append_kernel<<<blocks, threads, 0, st>>>(
         slot_k(c, slot), slot_v(c, slot), static_cast<const uint16_t*>(k_new),
         static_cast<const uint16_t*>(v_new), c->d_lens, batch, c->cfg.n_kv_heads, c->cfg.max_seq,
-        c->cfg.head_dim, c->cfg.stream_sink);
+        c->cfg.head_dim, c->cfg.stream_sink, c->d_pt, c->pt_stride, c->page_shift);
     return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
 }
 
@@ -444,15 +541,18 @@ int step_with_graph(lckv_cache* c, const void* const* q, void* const* out, const
 int run_step(lckv_cache* c, const void* const* q, void* const* out, const void* const* kn,
              const void* const* vn, int batch, cudaStream_t st)
 {
+    if (int rc = ensure_pages(c, batch, 1)) return rc;   // room for this step's token
+    if (int rc = sync_page_table(c, st)) return rc;
     const int rc = c->cfg.use_graph ? step_with_graph(c, q, out, kn, vn, batch, st)
                                     : enqueue_step(c, q, out, kn, vn, batch, st);
     if (rc == LCKV_OK) mirror_advance(c, batch);
     return rc;
 }
 
-int prefill_check(const lckv_cache* c, int n_max, int batch)
+int prefill_check(const lckv_cache* c, int n_max, int batch, bool attention)
 {
-    if (c->cfg.stream_sink > 0 || c->tm_pf_k.empty()) return LCKV_EINVAL;
+    if (c->cfg.stream_sink > 0) return LCKV_EINVAL;
+    if (attention && c->tm_pf_k.empty()) return LCKV_EINVAL;  // paged slots: write only
     if (batch < 1 || batch > c->cfg.max_batch || n_max < 1) return LCKV_EINVAL;
     for (int b = 0; b < batch; ++b)
         if (c->h_lens[b] > n_max) return LCKV_EINVAL;
@@ -467,7 +567,7 @@ int launch_prefill_write(lckv_cache* c, int slot, const void* k, const void* v, 
     lckv::prefill_write_kv_kernel<<<(unsigned)((n + threads - 1) / threads), threads, 0, st>>>(
         slot_k(c, slot), slot_v(c, slot), static_cast<const uint16_t*>(k),
         static_cast<const uint16_t*>(v), c->d_lens, batch, n_max, c->cfg.n_kv_heads, c->cfg.max_seq,
-        c->cfg.head_dim);
+        c->cfg.head_dim, c->d_pt, c->pt_stride, c->page_shift);
     return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
 }
 
@@ -618,6 +718,19 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     c->d_status = reinterpret_cast<int32_t*>(c->base + c->lay.off_status);
     c->d_partials = reinterpret_cast<float*>(c->base + c->lay.off_partials);
     c->h_lens.assign(cfg->max_batch, 0);
+    c->pt_stride = c->page_shift = 0;
+    c->d_pt = nullptr;
+    c->pt_dirty = false;
+    if (cfg->page_rows) {
+        c->pt_stride = (cfg->max_seq + cfg->page_rows - 1) / cfg->page_rows;
+        while ((1 << c->page_shift) < cfg->page_rows) ++c->page_shift;
+        c->d_pt = reinterpret_cast<int32_t*>(c->base + c->lay.off_pt);
+        c->h_pt.assign((size_t)cfg->max_batch * c->pt_stride, -1);
+        c->n_pages_of.assign(cfg->max_batch, 0);
+        c->free_pages.resize(cfg->n_pages);
+        for (int i = 0; i < cfg->n_pages; ++i) c->free_pages[i] = cfg->n_pages - 1 - i;  // pop gives 0, 1, ...
+        c->pt_dirty = true;
+    }
     {
         // About half of the L2 (measured optimum on B200, 126 MB L2: 60-70 MB; more than that and
         // the evict-last lines start displacing each other).  LCKV_L2_KEEP_MB overrides (0 = off).
@@ -636,7 +749,9 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     c->graph_exec = nullptr;
 
     if (c->kernel_kind == 2) {
-        const uint64_t rows = (uint64_t)cfg->max_batch * cfg->n_kv_heads * (uint64_t)cfg->max_seq;
+        const uint64_t rows = cfg->page_rows
+                                  ? (uint64_t)cfg->n_pages * cfg->n_kv_heads * (uint64_t)cfg->page_rows
+                                  : (uint64_t)cfg->max_batch * cfg->n_kv_heads * (uint64_t)cfg->max_seq;
         c->tm_k.resize(c->plan.n_slots);
         c->tm_v.resize(c->plan.n_slots);
         for (int s = 0; s < c->plan.n_slots; ++s) {
@@ -648,7 +763,7 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     {
         // prompt-encoding kernel: 64-row boxes over every slot (coordinates are 32-bit)
         const uint64_t rows = (uint64_t)cfg->max_batch * cfg->n_kv_heads * (uint64_t)cfg->max_seq;
-        if (rows < (1ull << 31)) {
+        if (rows < (1ull << 31) && cfg->page_rows == 0) {
             c->tm_pf_k.resize(c->plan.n_slots);
             c->tm_pf_v.resize(c->plan.n_slots);
             for (int s = 0; s < c->plan.n_slots; ++s) {
@@ -658,7 +773,19 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
             }
         }
     }
-    bool ok = cuda_ok(cudaFuncSetAttribute(lckv::prefill_tc5_kernel<128>,
+    bool ok = cuda_ok(cudaFuncSetAttribute(lckv::attn_alu_kernel<128, true>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           lckv::kAluSmemBytes)) &&
+              cuda_ok(cudaFuncSetAttribute(lckv::attn_alu_kernel<64, true>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           lckv::kAluSmemBytes)) &&
+              cuda_ok(cudaFuncSetAttribute(lckv::attn_mma_kernel<128, true>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           lckv::kMmaSmemBytes)) &&
+              cuda_ok(cudaFuncSetAttribute(lckv::attn_mma_kernel<64, true>,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           lckv::kMmaSmemBytes)) &&
+              cuda_ok(cudaFuncSetAttribute(lckv::prefill_tc5_kernel<128>,
                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            lckv::tc5_smem_bytes<128>())) &&
               cuda_ok(cudaFuncSetAttribute(lckv::prefill_tc5_kernel<64>,
@@ -721,6 +848,7 @@ int lckv_cache_reset(lckv_cache_t* c, const int32_t* host_lens, int32_t batch, v
             if (host_lens[b] < 0) return LCKV_EINVAL;
             if (host_lens[b] > c->cfg.max_seq && c->cfg.stream_sink == 0) return LCKV_ECAPACITY;
         }
+        if (int rc = repage(c, host_lens, batch)) return rc;
         for (int b = 0; b < batch; ++b) c->h_lens[b] = host_lens[b];
         // h_lens is the staging source: it lives as long as the cache and pageable copies are
         // staged before the call returns.
@@ -728,12 +856,13 @@ int lckv_cache_reset(lckv_cache_t* c, const int32_t* host_lens, int32_t batch, v
                                      cudaMemcpyHostToDevice, st)))
             return LCKV_ECUDA;
     } else {
+        if (int rc = repage(c, nullptr, batch)) return rc;
         for (int b = 0; b < batch; ++b) c->h_lens[b] = 0;
         if (!cuda_ok(cudaMemsetAsync(c->d_lens, 0, (size_t)batch * 4, st))) return LCKV_ECUDA;
     }
     if (!cuda_ok(cudaMemsetAsync(c->d_counters, 0, 2 * (size_t)c->n_workers * 4, st))) return LCKV_ECUDA;
     if (!cuda_ok(cudaMemsetAsync(c->d_status, 0, 4, st))) return LCKV_ECUDA;
-    return LCKV_OK;
+    return sync_page_table(c, st);
 }
 
 int lckv_cache_lengths(const lckv_cache_t* c, int32_t* host_out, int32_t batch, void* stream)
@@ -762,6 +891,14 @@ int lckv_cache_slot_ptrs(const lckv_cache_t* c, int32_t slot, void** k, void** v
     return LCKV_OK;
 }
 
+int lckv_cache_page_table(const lckv_cache_t* c, int32_t* host_out, int32_t* entries_per_seq)
+{
+    if (!c || !entries_per_seq || !c->cfg.page_rows) return LCKV_EINVAL;
+    *entries_per_seq = c->pt_stride;
+    if (host_out) std::memcpy(host_out, c->h_pt.data(), c->h_pt.size() * 4);
+    return LCKV_OK;
+}
+
 int lckv_append_kv(lckv_cache_t* c, int32_t slot, const void* k_new, const void* v_new,
                    int32_t batch, int32_t advance_len, void* stream)
 {
@@ -769,6 +906,8 @@ int lckv_append_kv(lckv_cache_t* c, int32_t slot, const void* k_new, const void*
     if (slot < 0 || slot >= c->plan.n_slots) return LCKV_EINVAL;
     if (max_len(c, batch) + 1 > c->cfg.max_seq) return LCKV_ECAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (int rc = ensure_pages(c, batch, 1)) return rc;
+    if (int rc = sync_page_table(c, st)) return rc;
     if (int rc = launch_append(c, slot, k_new, v_new, batch, st)) return rc;
     if (advance_len) {
         if (int rc = launch_advance(c, batch, st)) return rc;
@@ -785,6 +924,8 @@ int lckv_decode_attention(lckv_cache_t* c, int32_t slot, int32_t mode, const voi
     if (mode != LCKV_MODE_CONDENSED && mode != LCKV_MODE_STANDARD) return LCKV_EINVAL;
     if (max_len(c, batch) + mode > c->cfg.max_seq) return LCKV_ECAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (int rc = ensure_pages(c, batch, mode)) return rc;
+    if (int rc = sync_page_table(c, st)) return rc;
     if (int rc = launch_plan(c, batch, st)) return rc;
     return launch_attention(c, slot, mode, q, out, lse, batch, st);
 }
@@ -855,7 +996,8 @@ int lckv_prefill_write_kv(lckv_cache_t* c, int32_t slot, const void* k, const vo
                           int32_t n_max, int32_t batch, void* stream)
 {
     if (!c || !k || !v || slot < 0 || slot >= c->plan.n_slots) return LCKV_EINVAL;
-    if (int rc = prefill_check(c, n_max, batch)) return rc;
+    if (int rc = prefill_check(c, n_max, batch, false)) return rc;
+    if (int rc = sync_page_table(c, static_cast<cudaStream_t>(stream))) return rc;
     return launch_prefill_write(c, slot, k, v, n_max, batch, static_cast<cudaStream_t>(stream));
 }
 
@@ -864,7 +1006,7 @@ int lckv_prefill_attention(lckv_cache_t* c, int32_t slot, int32_t mode, const vo
 {
     if (!c || !q || !out || slot < 0 || slot >= c->plan.n_slots) return LCKV_EINVAL;
     if (mode != LCKV_MODE_CONDENSED && mode != LCKV_MODE_STANDARD) return LCKV_EINVAL;
-    if (int rc = prefill_check(c, n_max, batch)) return rc;
+    if (int rc = prefill_check(c, n_max, batch, true)) return rc;
     return launch_prefill_attention(c, slot, mode, q, out, n_max, batch,
                                     static_cast<cudaStream_t>(stream));
 }
@@ -874,7 +1016,7 @@ int lckv_prefill_iteration(lckv_cache_t* c, const void* const* q_layers, void* c
                            int32_t batch, void* stream)
 {
     if (!c || !q_layers || !out_layers || !k_layers || !v_layers) return LCKV_EINVAL;
-    if (int rc = prefill_check(c, n_max, batch)) return rc;
+    if (int rc = prefill_check(c, n_max, batch, true)) return rc;
     const Plan& pl = c->plan;
     const int L = c->cfg.n_layers;
     for (int l = 0; l < L; ++l) {
@@ -1023,6 +1165,9 @@ extern "C" int lckv_decode_attention_static(const void* k, const void* v, const 
     p.out_f32 = out_dtype;
     p.early_kv = 0;
     p.l2_keep = 0.f;
+    p.page_table = nullptr;
+    p.pt_stride = 0;
+    p.page_shift = 0;
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
     p.scale_log2 = scale * 1.4426950408889634f;
     if (head_dim == 128)

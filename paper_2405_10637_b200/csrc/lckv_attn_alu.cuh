@@ -49,6 +49,9 @@ struct AttnParams {
     int64_t T_cap;
     int32_t B, H_q, H_kv, mode, n_workers, out_f32;
     float scale_log2;         // softmax scale * log2(e)
+    const int32_t* page_table; // paged caches: [B_max][pt_stride] page ids (shared by all slots), else null
+    int32_t pt_stride;        // page-table entries per sequence
+    int32_t page_shift;       // log2(rows per page)
     float l2_keep;            // fraction of the cache lines to keep in L2 for the next layer's
                               // pass over the same cache (0: stream everything)
     int32_t early_kv;         // 1: the launcher guarantees that the plan tables and the visible K/V
@@ -81,7 +84,27 @@ __device__ __forceinline__ void cursor_next(TileCursor& c, const AttnParams& p, 
     } while (c.nt == 0);
 }
 
-template <int D>
+// Paged caches: a slot is [n_pages, H_kv, page_rows, D]; logical row r of sequence b lives in page
+// page_table[b][r / page_rows].  A tile never straddles pages (page_rows is a multiple of the tile).
+// The walker keeps the current page id and prefetches the next one, so the table look-up is off
+// the copy-issue path except at the first tile of a sequence.
+struct PageWalker {
+    int32_t b = -1, pg = -1, id = 0, next = 0;
+    __device__ __forceinline__ int64_t row(const AttnParams& p, int bb, int kvh, int r0)
+    {
+        const int q = r0 >> p.page_shift;
+        if (bb != b || q != pg) {
+            const int32_t* t = p.page_table + (size_t)bb * p.pt_stride;
+            id = (bb == b && q == pg + 1) ? next : __ldg(t + q);
+            next = (q + 1 < p.pt_stride) ? __ldg(t + q + 1) : 0;
+            b = bb;
+            pg = q;
+        }
+        return (((int64_t)id * p.H_kv + kvh) << p.page_shift) + (r0 & ((1 << p.page_shift) - 1));
+    }
+};
+
+template <int D, bool PAGED = false>
 __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnParams p)
 {
     constexpr int R = kAluSlotBytes / (D * 2);  // rows per tile: 16 (D=128), 32 (D=64)
@@ -130,13 +153,18 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
     TileCursor ci = cc;
 
     const uint64_t l2pol = make_l2_policy(p.l2_keep);
+    PageWalker walker;
     uint32_t issued = 0, islot = 0;
     auto issue = [&]() {
         const int rows = min(R, ci.nv - (int)ci.t * R);
         const uint32_t bytes = (uint32_t)rows * (D * 2);
         const uint16_t* base = (issued & 1) ? p.V : p.K;
-        const uint16_t* src =
-            base + (((int64_t)ci.b * p.H_kv + ci.h / g) * p.T_cap + (int64_t)ci.t * R) * D;
+        int64_t first_row;
+        if constexpr (PAGED)
+            first_row = walker.row(p, ci.b, ci.h / g, (int)ci.t * R);
+        else
+            first_row = ((int64_t)ci.b * p.H_kv + ci.h / g) * p.T_cap + (int64_t)ci.t * R;
+        const uint16_t* src = base + first_row * D;
         if (lane == 0) {
             mbar_expect_tx(bars + 8 * islot, bytes);
             bulk_g2s_hint(ring + islot * kAluSlotBytes, src, bytes, bars + 8 * islot, l2pol);

@@ -119,7 +119,7 @@ struct MmaParams {
     int32_t groups_per_kv;  // groups of 8 query heads that share one kv head
 };
 
-template <int D>
+template <int D, bool PAGED = false>
 __global__ void __launch_bounds__(kMmaWarps * 32, 1)
 attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV)
@@ -174,8 +174,11 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
 
     const uint64_t l2pol = make_l2_policy(p.l2_keep);
     uint32_t issued = 0, islot = 0;
+    PageWalker walker;
     auto issue = [&]() {
-        const int64_t row = ci.row;
+        int64_t row;
+        if constexpr (PAGED) row = walker.row(p, ci.b, ci.kvh, (int)ci.t * R);
+        else row = ci.row;
         if (lane == 0) {
             const void* tm = (issued & 1) ? (const void*)&tmV : (const void*)&tmK;
             mbar_expect_tx(bars + 8 * islot, kMmaSlotBytes);

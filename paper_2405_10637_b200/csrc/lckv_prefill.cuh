@@ -240,7 +240,8 @@ prefill_attn_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap t
 __global__ void prefill_write_kv_kernel(uint16_t* __restrict__ K, uint16_t* __restrict__ V,
                                         const uint16_t* __restrict__ k, const uint16_t* __restrict__ v,
                                         const int32_t* __restrict__ lens, int B, int n_max, int H_kv,
-                                        int64_t T_cap, int D)
+                                        int64_t T_cap, int D, const int32_t* __restrict__ page_table,
+                                        int pt_stride, int page_shift)
 {
     const int chunks = D / 8;
     const int64_t n = (int64_t)B * n_max * H_kv * chunks;
@@ -251,7 +252,12 @@ __global__ void prefill_write_kv_kernel(uint16_t* __restrict__ K, uint16_t* __re
     const int tok = (int)((i / ((int64_t)chunks * H_kv)) % n_max);
     const int b = (int)(i / ((int64_t)chunks * H_kv * n_max));
     if (tok >= lens[b] || tok >= T_cap) return;
-    const int64_t dst = ((((int64_t)b * H_kv + hh) * T_cap) + tok) * D + c * 8;
+    int64_t dst_row = (((int64_t)b * H_kv + hh) * T_cap) + tok;
+    if (page_table) {
+        const int64_t id = page_table[(int64_t)b * pt_stride + (tok >> page_shift)];
+        dst_row = ((id * H_kv + hh) << page_shift) + (tok & ((1 << page_shift) - 1));
+    }
+    const int64_t dst = dst_row * D + c * 8;
     const int64_t src = (((int64_t)b * n_max + tok) * H_kv + hh) * (int64_t)D + c * 8;
     *reinterpret_cast<uint4*>(K + dst) = *reinterpret_cast<const uint4*>(k + src);
     *reinterpret_cast<uint4*>(V + dst) = *reinterpret_cast<const uint4*>(v + src);

@@ -82,7 +82,8 @@ __global__ void append_kernel(uint16_t* __restrict__ K, uint16_t* __restrict__ V
                               const uint16_t* __restrict__ k_new,
                               const uint16_t* __restrict__ v_new,
                               const int32_t* __restrict__ lens, int B, int H_kv, int64_t T_cap,
-                              int D, int n_sink)
+                              int D, int n_sink, const int32_t* __restrict__ page_table,
+                              int pt_stride, int page_shift)
 {
     const int chunks = D / 8;
     const int64_t n = (int64_t)B * H_kv * chunks;
@@ -95,7 +96,12 @@ __global__ void append_kernel(uint16_t* __restrict__ K, uint16_t* __restrict__ V
     // Streaming mode: the first n_sink rows stay, the others form a ring of the most recent tokens.
     if (n_sink > 0 && row >= T_cap) row = n_sink + (row - n_sink) % (T_cap - n_sink);
     if (row < 0 || row >= T_cap) return;  // the host refuses such calls; never write out of range
-    const int64_t dst = (bh * T_cap + row) * D + c * 8;
+    int64_t dst_row = bh * T_cap + row;
+    if (page_table) {   // paged slot [n_pages, H_kv, page_rows, D]
+        const int64_t id = page_table[(int64_t)b * pt_stride + (row >> page_shift)];
+        dst_row = ((id * H_kv + (bh % H_kv)) << page_shift) + (row & ((1 << page_shift) - 1));
+    }
+    const int64_t dst = dst_row * D + c * 8;
     const int64_t src = bh * D + c * 8;
     *reinterpret_cast<uint4*>(K + dst) = *reinterpret_cast<const uint4*>(k_new + src);
     *reinterpret_cast<uint4*>(V + dst) = *reinterpret_cast<const uint4*>(v_new + src);

@@ -39,7 +39,7 @@ class Case:
 
     def __init__(self, L, w, Hq, Hkv, d, lens, T_cap, variant=0, out_dtype=0, seed=1234, std=1.0,
                  poison=True, B_max=None, scale=0.0, kernel_kind=0, host_staging=0, use_graph=0,
-                 stream_sink=0):
+                 stream_sink=0, page_rows=0, n_pages=0):
         self.L, self.w, self.Hq, self.Hkv, self.d = L, w, Hq, Hkv, d
         self.lens = np.asarray(lens, np.int32).copy()
         self.B = len(lens)
@@ -48,14 +48,20 @@ class Case:
         self.cfg = lk.make_config(L, w, Hq, Hkv, d, B_max, T_cap, softmax_scale=scale,
                                   top_variant=variant, out_dtype=out_dtype, kernel_kind=kernel_kind,
                                   host_staging=host_staging, use_graph=use_graph,
-                                  stream_sink=stream_sink)
+                                  stream_sink=stream_sink, page_rows=page_rows, n_pages=n_pages)
         self.stream_sink = stream_sink
+        self.page_rows = page_rows
         self.scale = scale if scale > 0 else d ** -0.5
         self.cache = lk.Cache(self.cfg)
         self.plan = orc.plan(L, w, variant)
         self.n_slots = self.plan["n_slots"]
         assert self.cache.info.n_slots == self.n_slots
         self.hK, self.hV = [], []
+        if page_rows:
+            # pages are assigned on reset; a first reset with the lengths reversed leaves the free
+            # list in a different order, so the final assignment is not simply 0, 1, 2, ...
+            self.cache.lckv_cache_reset(self.lens[::-1].tolist())
+            self.cache.lckv_cache_reset(self.lens.tolist())
         for s in range(self.n_slots):
             kb = syn.bits(syn.randn_bf16((B_max, Hkv, T_cap, d), seed + 2 * s, std=std))
             vb = syn.bits(syn.randn_bf16((B_max, Hkv, T_cap, d), seed + 2 * s + 1, std=std))
@@ -65,9 +71,15 @@ class Case:
                     kb[b, :, n:] = NAN_BITS
                     vb[b, :, n:] = NAN_BITS
             kt, vt = self.cache.slot_tensors(s)
-            kt.copy_(syn.from_bits(kb)); vt.copy_(syn.from_bits(vb))
+            if page_rows:
+                kt.copy_(syn.from_bits(np.full(tuple(kt.shape), NAN_BITS, np.uint16)))
+                vt.copy_(kt)
+                self._scatter(kt, kb); self._scatter(vt, vb)
+            else:
+                kt.copy_(syn.from_bits(kb)); vt.copy_(syn.from_bits(vb))
             self.hK.append(kb); self.hV.append(vb)
-        self.cache.lckv_cache_reset(self.lens.tolist())
+        if not page_rows:
+            self.cache.lckv_cache_reset(self.lens.tolist())
         self.step_no = 0
 
     def step_inputs(self):
@@ -124,11 +136,39 @@ class Case:
             self.check_state()
         return outs, want, stats
 
+    def _scatter(self, pool, logical_bits):
+        """Paged cache: copy the logical rows [B, Hkv, T_cap, d] into the pages each sequence owns."""
+        P = self.page_rows
+        pt = self.cache.lckv_cache_page_table()
+        for b in range(pt.shape[0]):
+            for i in range(pt.shape[1]):
+                pg = int(pt[b, i])
+                if pg < 0:
+                    break
+                rows = logical_bits[b, :, i * P:(i + 1) * P]
+                pool[pg, :, :rows.shape[1]].copy_(syn.from_bits(rows))
+
+    def _gather(self, pool, b):
+        """Paged cache: the logical rows sequence b owns, [Hkv, n_owned_rows, d] as bits."""
+        pt = self.cache.lckv_cache_page_table()
+        pages = [int(x) for x in pt[b] if int(x) >= 0]
+        if not pages:
+            return np.zeros((self.Hkv, 0, self.d), np.uint16)
+        return np.concatenate([syn.bits(pool[pg]) for pg in pages], axis=1)
+
     def check_state(self):
         """Lengths and every byte of every cache, bit for bit."""
         assert self.cache.lckv_cache_lengths(self.B) == self.lens.tolist()
         for s in range(self.n_slots):
             kt, vt = self.cache.slot_tensors(s)
+            if self.page_rows:
+                for b in range(self.B):
+                    gk, gv = self._gather(kt, b), self._gather(vt, b)
+                    n = min(gk.shape[1], self.T_cap)
+                    assert n >= min(int(self.lens[b]), self.T_cap)
+                    assert np.array_equal(gk[:, :n], self.hK[s][b][:, :n]), f"slot {s} seq {b} K differs"
+                    assert np.array_equal(gv[:, :n], self.hV[s][b][:, :n]), f"slot {s} seq {b} V differs"
+                continue
             assert np.array_equal(syn.bits(kt), self.hK[s]), f"slot {s} K differs"
             assert np.array_equal(syn.bits(vt), self.hV[s]), f"slot {s} V differs"
 

@@ -333,3 +333,50 @@ def test_a_sequence_does_not_depend_on_its_batch_mates():
     torch.cuda.synchronize()
     assert (a5[:2] - a2).abs().max().item() < 1e-5
     cache.close()
+
+
+# ---- paged caches ---------------------------------------------------------------------------------
+
+@pytest.mark.parametrize("shape", ["mha128", "mha64", "gqa64", "gqa128"])
+def test_paged_cache_matches_oracle(shape):
+    """Slots as pools of 64-row pages: a sequence owns ceil(len / 64) pages, assigned in a scrambled
+    order; decode steps that cross page boundaries (new pages taken from the pool) stay exact."""
+    kw = {"mha128": dict(Hq=4, Hkv=4, d=128, std=1.0), "mha64": dict(Hq=4, Hkv=4, d=64, std=1.0),
+          "gqa64": dict(Hq=16, Hkv=2, d=64, std=0.25), "gqa128": dict(Hq=8, Hkv=1, d=128, std=0.25)}[shape]
+    lens = [0, 1, 63, 64, 65, 127, 128, 300, 500, 62]
+    c = Case(L=4, w=2, lens=lens, T_cap=520, seed=123, page_rows=64, n_pages=40, **kw)
+    pt0 = c.cache.lckv_cache_page_table()
+    assert [(int((pt0[b] >= 0).sum())) for b in range(len(lens))] == [(n + 63) // 64 for n in lens]
+    for _ in range(4):
+        c.step()
+    pt = c.cache.lckv_cache_page_table()
+    assert [(int((pt[b] >= 0).sum())) for b in range(len(lens))] == [(n + 4 + 63) // 64 for n in lens]
+    used = pt[pt >= 0].tolist()
+    assert len(used) == len(set(used)), "a page is owned twice"
+    c.close()
+
+
+def test_paged_cache_pool_exhaustion_and_reuse():
+    B, H, d = 3, 2, 64
+    cfg = lk.make_config(2, 0, H, H, d, B, 256, page_rows=64, n_pages=4)
+    cache = lk.Cache(cfg)
+    with pytest.raises(lk.LckvError) as e:
+        cache.lckv_cache_reset([100, 100, 100])            # needs 6 pages
+    assert e.value.status == lk.ECAPACITY
+    cache.lckv_cache_reset([64, 64, 100])                  # 1 + 1 + 2 pages: pool full
+    dev = cache.device
+    x = torch.zeros((B, H, d), dtype=torch.bfloat16, device=dev)
+    with pytest.raises(lk.LckvError) as e:                  # rows 64 need a new page each: none left
+        cache.lckv_layer_stack_step([x, x], [x.clone(), x.clone()], [None, x], [None, x])
+    assert e.value.status == lk.ECAPACITY
+    assert cache.lckv_cache_lengths(B) == [64, 64, 100]
+    pt = cache.lckv_cache_page_table()
+    assert int((pt >= 0).sum()) == 4
+    cache.lckv_cache_reset([10, 0, 0])                     # pages go back to the pool
+    assert int((cache.lckv_cache_page_table() >= 0).sum()) == 1
+    cache.lckv_layer_stack_step([x, x], [x.clone(), x.clone()], [None, x], [None, x])
+    torch.cuda.synchronize()
+    assert cache.lckv_cache_lengths(B) == [11, 1, 1]
+    cache.close()
+    bad = lk.make_config(2, 0, H, H, d, B, 256, page_rows=48, n_pages=4)   # not a power of two
+    assert lk.lckv_cache_bytes(bad) == 0
