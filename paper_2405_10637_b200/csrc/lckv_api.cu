@@ -552,7 +552,7 @@ int run_step(lckv_cache* c, const void* const* q, void* const* out, const void* 
 int prefill_check(const lckv_cache* c, int n_max, int batch, bool attention)
 {
     if (c->cfg.stream_sink > 0) return LCKV_EINVAL;
-    if (attention && c->tm_pf_k.empty()) return LCKV_EINVAL;  // paged slots: write only
+    if (attention && c->tm_pf_k.empty()) return LCKV_EINVAL;  // slot too large for 32-bit TMA rows
     if (batch < 1 || batch > c->cfg.max_batch || n_max < 1) return LCKV_EINVAL;
     for (int b = 0; b < batch; ++b)
         if (c->h_lens[b] > n_max) return LCKV_EINVAL;
@@ -587,6 +587,9 @@ int launch_prefill_attention(lckv_cache* c, int slot, int mode, const void* q, v
     p.mode = mode;
     p.out_f32 = c->cfg.out_dtype;
     p.scale_log2 = c->scale_log2;
+    p.page_table = c->d_pt;
+    p.pt_stride = c->pt_stride;
+    p.page_shift = c->page_shift;
     int longest = 0;
     for (int b = 0; b < batch; ++b) longest = c->h_lens[b] > longest ? c->h_lens[b] : longest;
     if (longest == 0) return LCKV_OK;
@@ -762,8 +765,10 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     }
     {
         // prompt-encoding kernel: 64-row boxes over every slot (coordinates are 32-bit)
-        const uint64_t rows = (uint64_t)cfg->max_batch * cfg->n_kv_heads * (uint64_t)cfg->max_seq;
-        if (rows < (1ull << 31) && cfg->page_rows == 0) {
+        const uint64_t rows = cfg->page_rows
+                                  ? (uint64_t)cfg->n_pages * cfg->n_kv_heads * (uint64_t)cfg->page_rows
+                                  : (uint64_t)cfg->max_batch * cfg->n_kv_heads * (uint64_t)cfg->max_seq;
+        if (rows < (1ull << 31)) {
             c->tm_pf_k.resize(c->plan.n_slots);
             c->tm_pf_v.resize(c->plan.n_slots);
             for (int s = 0; s < c->plan.n_slots; ++s) {
@@ -1007,6 +1012,7 @@ int lckv_prefill_attention(lckv_cache_t* c, int32_t slot, int32_t mode, const vo
     if (!c || !q || !out || slot < 0 || slot >= c->plan.n_slots) return LCKV_EINVAL;
     if (mode != LCKV_MODE_CONDENSED && mode != LCKV_MODE_STANDARD) return LCKV_EINVAL;
     if (int rc = prefill_check(c, n_max, batch, true)) return rc;
+    if (int rc = sync_page_table(c, static_cast<cudaStream_t>(stream))) return rc;
     return launch_prefill_attention(c, slot, mode, q, out, n_max, batch,
                                     static_cast<cudaStream_t>(stream));
 }
@@ -1024,6 +1030,7 @@ int lckv_prefill_iteration(lckv_cache_t* c, const void* const* q_layers, void* c
         if (pl.write_slot[l] >= 0 && (!k_layers[l] || !v_layers[l])) return LCKV_EINVAL;
     }
     cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (int rc = sync_page_table(c, st)) return rc;
     for (int l = 0; l < L; ++l) {
         if (pl.write_slot[l] >= 0 && pl.write_before[l])
             if (int rc = launch_prefill_write(c, pl.write_slot[l], k_layers[l], v_layers[l], n_max, batch, st))

@@ -31,7 +31,21 @@ struct PrefillParams {
     int64_t T_cap;
     int32_t B, n_max, H_q, H_kv, mode, out_f32;
     float scale_log2;
+    const int32_t* page_table;  // paged slots: [B_max][pt_stride] page ids, else null
+    int32_t pt_stride, page_shift;
 };
+
+// First cache row (of the 2-D [rows, D] view of a slot) of the 64-row tile jt of (b, kv head).
+__device__ __forceinline__ int64_t prefill_tile_row(const PrefillParams& p, int b, int kvh, int jt,
+                                                    int tile_rows)
+{
+    const int r0 = jt * tile_rows;
+    if (p.page_table) {   // a tile never straddles pages: the page size is a multiple of 64
+        const int64_t id = __ldg(p.page_table + (size_t)b * p.pt_stride + (r0 >> p.page_shift));
+        return ((id * p.H_kv + kvh) << p.page_shift) + (r0 & ((1 << p.page_shift) - 1));
+    }
+    return ((int64_t)b * p.H_kv + kvh) * p.T_cap + r0;
+}
 
 template <int D>
 __global__ void __launch_bounds__(kPfWarps * 32)
@@ -50,7 +64,7 @@ prefill_attn_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap t
     const int nb = min(__ldg(p.lens + b), p.n_max);
     if (mb * kPfBM >= nb) return;
     const int g = p.H_q / p.H_kv;
-    const int64_t row0 = ((int64_t)b * p.H_kv + h / g) * p.T_cap;
+    const int kvh = h / g;
     const int n_kv = mb + 1;             // tiles 0 .. mb reach the diagonal
 
     extern __shared__ uint8_t smem_raw[];
@@ -67,11 +81,12 @@ prefill_attn_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap t
     auto issue = [&](int jt) {  // thread 0 only
         const int s = jt & 1;
         const uint32_t kb = smem0 + s * 2 * TILEB, vb = kb + TILEB;
+        const int32_t row = (int32_t)prefill_tile_row(p, b, kvh, jt, kPfBN);
         mbar_expect_tx(bars + 8 * s, 2 * TILEB);
 #pragma unroll
         for (int bx = 0; bx < NBOX; ++bx) {
-            tma_load_2d(kb + bx * BOXB, &tmK, bx * 64, (int32_t)(row0 + (int64_t)jt * kPfBN), bars + 8 * s);
-            tma_load_2d(vb + bx * BOXB, &tmV, bx * 64, (int32_t)(row0 + (int64_t)jt * kPfBN), bars + 8 * s);
+            tma_load_2d(kb + bx * BOXB, &tmK, bx * 64, row, bars + 8 * s);
+            tma_load_2d(vb + bx * BOXB, &tmV, bx * 64, row, bars + 8 * s);
         }
     };
     if (tid == 0) issue(0);

@@ -174,7 +174,7 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
     const int nb = min(__ldg(p.lens + b), p.n_max);
     if (mb * kT5BM >= nb) return;
     const int g = p.H_q / p.H_kv;
-    const int64_t row0 = ((int64_t)b * p.H_kv + h / g) * p.T_cap;
+    const int kvh = h / g;
     const int i_max = min(mb * kT5BM + kT5BM - 1, nb - 1);
     const int c_last = i_max - 1 + p.mode;         // last cache row any query of this block sees
     const int n_kv = c_last < 0 ? 0 : c_last / kT5BN + 1;
@@ -231,18 +231,17 @@ prefill_tc5_kernel(const PrefillParams p, const __grid_constant__ CUtensorMap tm
                 const uint32_t par_prev = ((j >> 1) - 1) & 1;
                 if (j >= 2) ok = mbar_wait_bounded(bKe + 8 * st, par_prev, kT5WaitLimit);
                 if (!ok) break;
+                const int32_t row = (int32_t)prefill_tile_row(p, b, kvh, j, kT5BN);
                 mbar_expect_tx(bKf + 8 * st, KV_BYTES);
 #pragma unroll
                 for (int bx = 0; bx < NBOX; ++bx)
-                    tma_load_2d(sK + st * KV_BYTES + bx * KBOX, &tmK, bx * 64,
-                                (int32_t)(row0 + (int64_t)j * kT5BN), bKf + 8 * st);
+                    tma_load_2d(sK + st * KV_BYTES + bx * KBOX, &tmK, bx * 64, row, bKf + 8 * st);
                 if (j >= 2) ok = mbar_wait_bounded(bVe + 8 * st, par_prev, kT5WaitLimit);
                 if (!ok) break;
                 mbar_expect_tx(bVf + 8 * st, KV_BYTES);
 #pragma unroll
                 for (int bx = 0; bx < NBOX; ++bx)
-                    tma_load_2d(sV + st * KV_BYTES + bx * KBOX, &tmV, bx * 64,
-                                (int32_t)(row0 + (int64_t)j * kT5BN), bVf + 8 * st);
+                    tma_load_2d(sV + st * KV_BYTES + bx * KBOX, &tmV, bx * 64, row, bVf + 8 * st);
             }
             if (!ok) atomicExch(p.status, kStatusTimeout);
         }

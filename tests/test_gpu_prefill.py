@@ -161,3 +161,36 @@ def test_prefill_errors():
         c2.lckv_prefill_attention(0, 0, q)
     assert e.value.status == lk.EINVAL
     c2.close()
+
+
+@pytest.mark.parametrize("kernel", ["tc5", "mma"])
+def test_prefill_on_paged_cache(kernel, monkeypatch):
+    """Prompt encoding over slots made of 64-row pages (scrambled page order), both kernels."""
+    from helpers import Case
+    monkeypatch.setenv("LCKV_PREFILL_KERNEL", kernel)
+    lens = [130, 64, 1, 200, 65]
+    c = Case(L=4, w=2, Hq=8, Hkv=2, d=64, lens=lens, T_cap=256, seed=17, std=0.5, page_rows=64, n_pages=14)
+    dev, B, n_max = c.cache.device, len(lens), 200
+    plan = c.plan
+    for it in range(2):
+        q = [syn.randn_bf16((B, n_max, c.Hq, c.d), 300 + 10 * it + l, std=0.5) for l in range(c.L)]
+        k = [syn.randn_bf16((B, n_max, c.Hkv, c.d), 400 + 10 * it + l, std=0.5)
+             if plan["write_slot"][l] >= 0 else None for l in range(c.L)]
+        v = [syn.randn_bf16((B, n_max, c.Hkv, c.d), 500 + 10 * it + l, std=0.5)
+             if plan["write_slot"][l] >= 0 else None for l in range(c.L)]
+        outs = [torch.zeros((B, n_max, c.Hq, c.d), dtype=torch.bfloat16, device=dev) for _ in range(c.L)]
+        c.cache.lckv_prefill_iteration([t.to(dev) for t in q], outs,
+                                       [None if t is None else t.to(dev) for t in k],
+                                       [None if t is None else t.to(dev) for t in v])
+        torch.cuda.synchronize()
+        assert c.cache.lckv_cache_status() == 0
+        want = orc.prefill_iteration(c.L, c.w, [syn.bits(t) for t in q],
+                                     [None if t is None else syn.bits(t) for t in k],
+                                     [None if t is None else syn.bits(t) for t in v],
+                                     c.hK, c.hV, c.lens, c.scale)
+        for l in range(c.L):
+            for b, nb in enumerate(lens):
+                compare(outs[l][b, :nb], want[l][b, :nb], f"iteration {it} layer {l} seq {b}")
+        c.check_state()
+    c.step()   # and decoding continues on the same pages
+    c.close()
