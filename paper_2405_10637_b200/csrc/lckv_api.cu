@@ -706,7 +706,7 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     c->grid = sm;
     c->n_workers = sm * workers_per_sm(*cfg);
     c->kernel_kind = resolve_kernel_kind(*cfg);
-    c->rows_per_tile = lckv::kAluSlotBytes / (cfg->head_dim * 2);
+    c->rows_per_tile = (c->kernel_kind == 2 ? lckv::kMmaSlotBytes : lckv::kAluSlotBytes) / (cfg->head_dim * 2);
     c->h_pairs = c->kernel_kind == 2 ? cfg->n_q_heads / 8 : cfg->n_q_heads;
     make_layout(*cfg, c->plan.n_slots, c->n_workers, c->n_kv_layers, c->lay);
     if (dev_bytes < c->lay.total_bytes) { delete c; return LCKV_ENOMEM; }

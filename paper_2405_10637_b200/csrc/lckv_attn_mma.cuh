@@ -21,11 +21,14 @@ namespace lckv {
 #define LCKV_MMA_WARPS 8
 #endif
 #ifndef LCKV_MMA_SLOTS
-#define LCKV_MMA_SLOTS 3
+#define LCKV_MMA_SLOTS 2
 #endif
 constexpr int kMmaWarps = LCKV_MMA_WARPS;
 constexpr int kMmaSlots = LCKV_MMA_SLOTS;
-constexpr int kMmaSlotBytes = 4096;
+#ifndef LCKV_MMA_SLOT_BYTES
+#define LCKV_MMA_SLOT_BYTES 8192
+#endif
+constexpr int kMmaSlotBytes = LCKV_MMA_SLOT_BYTES;
 constexpr int kMmaSmemBytes = kMmaWarps * kMmaSlots * (kMmaSlotBytes + 8) + 1024;  // + alignment slack
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
