@@ -23,15 +23,18 @@ namespace lckv {
 #ifndef LCKV_ALU_WARPS
 #define LCKV_ALU_WARPS 8
 #endif
+#ifndef LCKV_ALU_SLOT_BYTES
+#define LCKV_ALU_SLOT_BYTES 8192
+#endif
 #ifndef LCKV_ALU_SLOTS
-#define LCKV_ALU_SLOTS 4
+#define LCKV_ALU_SLOTS 2
 #endif
 #ifndef LCKV_ALU_FFMA2
 #define LCKV_ALU_FFMA2 1
 #endif
 constexpr int kAluWarps = LCKV_ALU_WARPS;  // workers per CTA
 constexpr int kAluSlots = LCKV_ALU_SLOTS;  // ring slots per worker
-constexpr int kAluSlotBytes = 4096;  // one tile of K or of V
+constexpr int kAluSlotBytes = LCKV_ALU_SLOT_BYTES;  // one tile of K or of V (a multiple of 4 KB)
 constexpr int kAluSmemBytes = kAluWarps * kAluSlots * (kAluSlotBytes + 8);
 
 struct AttnParams {
@@ -107,10 +110,12 @@ struct PageWalker {
 template <int D, bool PAGED = false>
 __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnParams p)
 {
-    constexpr int R = kAluSlotBytes / (D * 2);  // rows per tile: 16 (D=128), 32 (D=64)
+    constexpr int SUB = kAluSlotBytes / 4096;   // 4 KB sub-tiles per tile
+    constexpr int R1 = 4096 / (D * 2);          // rows per sub-tile: 16 (D=128), 32 (D=64)
+    constexpr int R = SUB * R1;                 // rows per tile
     constexpr int LPR = D / 8;                  // lanes per row (16 bytes each)
     constexpr int RPI = 32 / LPR;               // rows covered by one warp-wide 16-byte load
-    constexpr int NP = R / RPI;                 // such loads per tile = partial sums per lane
+    constexpr int NP = R1 / RPI;                // such loads per sub-tile = partial sums per lane
     constexpr int DUP = LPR / NP;               // lanes that end up holding the same score
     constexpr int NS = kAluSlots;
     constexpr int REC = D + 4;                  // floats per partial record
@@ -230,9 +235,10 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
 
         // ---- K tile: scores -----------------------------------------------------------------
         if (!mbar_wait_bounded(bars + 8 * cslot, cphase)) { ok = false; break; }
-        float part[NP];
-        {
-            const uint32_t base = ring + cslot * kAluSlotBytes + grp * (D * 2) + a * 16;
+        float part[SUB][NP];
+#pragma unroll
+        for (int u = 0; u < SUB; ++u) {
+            const uint32_t base = ring + cslot * kAluSlotBytes + u * 4096 + grp * (D * 2) + a * 16;
 #pragma unroll
             for (int i = 0; i < NP; ++i) {
                 const uint4 kv = lds128(base + i * (RPI * D * 2));
@@ -243,7 +249,7 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
                 acc = ffma2(pack_f32x2(bf16lo(kv.w), bf16hi(kv.w)), q2[3], acc);
                 float ax, ay;
                 unpack_f32x2(acc, ax, ay);
-                part[i] = ax + ay;
+                part[u][i] = ax + ay;
 #else
                 float s = bf16lo(kv.x) * qf[0];
                 s = fmaf(bf16hi(kv.x), qf[1], s);
@@ -253,7 +259,7 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
                 s = fmaf(bf16hi(kv.z), qf[5], s);
                 s = fmaf(bf16lo(kv.w), qf[6], s);
                 s = fmaf(bf16hi(kv.w), qf[7], s);
-                part[i] = s;
+                part[u][i] = s;
 #endif
             }
         }
@@ -264,41 +270,52 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
 
         // Sum each row's LPR partial dot products.  Exchange steps halve the number of values a
         // lane carries (8 -> 4 -> 2 -> 1); with 16 lanes per row one plain butterfly step remains.
-        {
+        // Afterwards this lane holds, per sub-tile, the score of load index a / DUP, i.e. of row:
+        const int my_row = (a / DUP) * RPI + grp;
+        float sc[SUB];
+#pragma unroll
+        for (int u = 0; u < SUB; ++u) {
+            float* pt = part[u];
             bool up = (a & (LPR / 2)) != 0;
 #pragma unroll
             for (int k = 0; k < 4; ++k) {
-                const float send = up ? part[k] : part[k + 4];
-                const float keep = up ? part[k + 4] : part[k];
-                part[k] = keep + __shfl_xor_sync(FULL, send, LPR / 2);
+                const float send = up ? pt[k] : pt[k + 4];
+                const float keep = up ? pt[k + 4] : pt[k];
+                pt[k] = keep + __shfl_xor_sync(FULL, send, LPR / 2);
             }
             up = (a & (LPR / 4)) != 0;
 #pragma unroll
             for (int k = 0; k < 2; ++k) {
-                const float send = up ? part[k] : part[k + 2];
-                const float keep = up ? part[k + 2] : part[k];
-                part[k] = keep + __shfl_xor_sync(FULL, send, LPR / 4);
+                const float send = up ? pt[k] : pt[k + 2];
+                const float keep = up ? pt[k + 2] : pt[k];
+                pt[k] = keep + __shfl_xor_sync(FULL, send, LPR / 4);
             }
             up = (a & (LPR / 8)) != 0;
             {
-                const float send = up ? part[0] : part[1];
-                const float keep = up ? part[1] : part[0];
-                part[0] = keep + __shfl_xor_sync(FULL, send, LPR / 8);
+                const float send = up ? pt[0] : pt[1];
+                const float keep = up ? pt[1] : pt[0];
+                pt[0] = keep + __shfl_xor_sync(FULL, send, LPR / 8);
             }
-            if (DUP == 2) part[0] += __shfl_xor_sync(FULL, part[0], 1);
+            if (DUP == 2) pt[0] += __shfl_xor_sync(FULL, pt[0], 1);
+            sc[u] = (u * R1 + my_row < rows) ? pt[0] : -INFINITY;
         }
-        // This lane now holds the score of load index a / DUP, i.e. of tile row:
-        const int my_row = (a / DUP) * RPI + grp;
-        const float s = (my_row < rows) ? part[0] : -INFINITY;
 
-        float m_tile = s;
+        float m_tile = sc[0];
+#pragma unroll
+        for (int u = 1; u < SUB; ++u) m_tile = fmaxf(m_tile, sc[u]);
 #pragma unroll
         for (int off = 16; off >= 1; off >>= 1)
             m_tile = fmaxf(m_tile, __shfl_xor_sync(FULL, m_tile, off));
         const float m_new = fmaxf(m_run, m_tile);
         const float alpha = ex2(m_run - m_new);
-        const float pr = ex2(s - m_new);
-        l_run = fmaf(l_run, alpha, pr);
+        float pr[SUB];
+        float p_sum = 0.f;
+#pragma unroll
+        for (int u = 0; u < SUB; ++u) {
+            pr[u] = ex2(sc[u] - m_new);
+            p_sum += pr[u];
+        }
+        l_run = fmaf(l_run, alpha, p_sum);
         m_run = m_new;
 #if LCKV_ALU_FFMA2
         {
@@ -322,11 +339,12 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
             fence_proxy_async_smem();
             __syncwarp();
         }
-        {
-            const uint32_t base = ring + cslot * kAluSlotBytes + grp * (D * 2) + a * 16;
+#pragma unroll
+        for (int u = 0; u < SUB; ++u) {
+            const uint32_t base = ring + cslot * kAluSlotBytes + u * 4096 + grp * (D * 2) + a * 16;
 #pragma unroll
             for (int i = 0; i < NP; ++i) {
-                const float pi = __shfl_sync(FULL, pr, grp * LPR + i * DUP);
+                const float pi = __shfl_sync(FULL, pr[u], grp * LPR + i * DUP);
                 const uint4 vv = lds128(base + i * (RPI * D * 2));
 #if LCKV_ALU_FFMA2
                 const uint64_t p2 = pack_f32x2(pi, pi);
