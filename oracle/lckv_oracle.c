@@ -15,7 +15,10 @@
  * Pins (see tests/): brute-force n x n masked attention written independently
  * in numpy, torch's scaled_dot_product_attention in float64 for w = L, closed
  * forms (q = 0, one visible key, empty visible set, dominant key), permutation
- * invariance, log-sum-exp merge of any partition, hand-enumerated warmup sets.
+ * invariance, log-sum-exp merge of any partition, hand-enumerated warmup sets;
+ * for the key/value producer: exact rational sums, selector weights, a library
+ * matmul, torch's bf16 rounding on exact products, the complex-number form of
+ * the rotary encoding and its relative-position property.
  *
  * Readings of the paper where it is silent (each one is a switch here):
  *   top_variant 0  the shared cache is the cache of layer L-1 itself, even
@@ -399,4 +402,82 @@ int lckv_oracle_prefill_iteration(int L, int w, int top_variant, const uint16_t*
                                               v_layers[l], lens, B, n_max, H_kv, T_cap, d);
     free(plan);
     return rc;
+}
+
+/* float64 -> bf16 bits, round to nearest, ties to even (the one rounding of a produced key or
+ * value on its way into the bf16 cache).  The value is first rounded to binary32 by the C
+ * conversion (itself to nearest even); double rounding cannot differ from direct rounding here
+ * except on exact binary32 ties, which the callers' magnitudes make measure-zero events, and the
+ * comparison that uses these bits allows one bf16 unit anyway. */
+static uint16_t f64_to_bf16(double x)
+{
+    float f = (float)x;
+    uint32_t u;
+    memcpy(&u, &f, sizeof u);
+    if ((u & 0x7fffffffu) > 0x7f800000u) return (uint16_t)((u >> 16) | 0x40u); /* NaN stays NaN */
+    uint32_t lsb = (u >> 16) & 1u;
+    u += 0x7fffu + lsb;
+    return (uint16_t)(u >> 16);
+}
+
+/*
+ * Keys and values of the new token (Section 2.1: W_K, W_V map a hidden representation to its key
+ * and value; in the condensed model only the layers that own a cache still do this):
+ *   k[b, f] = sum_c W_K[f, c] x[b, c],   v[b, f] = sum_c W_V[f, c] x[b, c],
+ *   x [B, d_model], W [H_kv * d, d_model] (row f = output feature, as a linear layer stores it),
+ *   feature f = kv head f / d, dimension f mod d.
+ * Optional position encoding of the key (the paper's models are Llama models, whose keys are
+ * rotated by their position before they are cached; the paper does not restate it, so it is a
+ * switch: cos == NULL leaves k as projected).  Rotary embedding in the half-split pairing: with
+ * p = lens[b] the token's position and i < d/2,
+ *   k'[i]       = k[i] cos[p, i] - k[i + d/2] sin[p, i]
+ *   k'[i + d/2] = k[i + d/2] cos[p, i] + k[i] sin[p, i].
+ * cos, sin [n_pos, d/2] are inputs (float32 values, widened exactly).
+ * Outputs: k_bits, v_bits [B, H_kv, d] bf16 (one rounding from float64); k_f64, v_f64 (optional)
+ * the unrounded values.
+ */
+int lckv_oracle_project_kv(const uint16_t* x, const uint16_t* w_k, const uint16_t* w_v,
+                           const float* cos_tab, const float* sin_tab, int n_pos,
+                           const int32_t* lens, int B, int H_kv, int d, int d_model,
+                           uint16_t* k_bits, uint16_t* v_bits, double* k_f64, double* v_f64)
+{
+    if (B < 1 || H_kv < 1 || d < 2 || (d & 1) || d_model < 1) return LCKV_ORACLE_EINVAL;
+    if ((cos_tab == NULL) != (sin_tab == NULL)) return LCKV_ORACLE_EINVAL;
+    const int half = d / 2;
+    if (cos_tab)
+        for (int b = 0; b < B; ++b)
+            if (lens[b] < 0 || lens[b] >= n_pos) return LCKV_ORACLE_EINVAL;
+    const int64_t F = (int64_t)H_kv * d;
+    double* kp = (double*)malloc(sizeof(double) * (size_t)((int64_t)B * F));   /* projected keys */
+    if (!kp) return LCKV_ORACLE_EINVAL;
+#pragma omp parallel for schedule(static)
+    for (int64_t bf = 0; bf < (int64_t)B * F; ++bf) {
+        const int64_t b = bf / F, f = bf % F;
+        double ks = 0.0, vs = 0.0;
+        for (int c = 0; c < d_model; ++c) {
+            const double xc = bf16_to_f64(x[b * d_model + c]);
+            ks += bf16_to_f64(w_k[f * d_model + c]) * xc;
+            vs += bf16_to_f64(w_v[f * d_model + c]) * xc;
+        }
+        kp[bf] = ks;
+        if (v_f64) v_f64[bf] = vs;
+        v_bits[bf] = f64_to_bf16(vs);
+    }
+    for (int64_t bh = 0; bh < (int64_t)B * H_kv; ++bh) {
+        const int64_t b = bh / H_kv;
+        const int64_t p = lens[b];
+        double* kh = kp + bh * d;                      /* one head of one sequence */
+        for (int i = 0; i < half && cos_tab; ++i) {
+            const double cs = (double)cos_tab[p * half + i], sn = (double)sin_tab[p * half + i];
+            const double lo = kh[i], hi = kh[i + half];
+            kh[i] = lo * cs - hi * sn;
+            kh[i + half] = hi * cs + lo * sn;
+        }
+        for (int i = 0; i < d; ++i) {
+            if (k_f64) k_f64[bh * d + i] = kh[i];
+            k_bits[bh * d + i] = f64_to_bf16(kh[i]);
+        }
+    }
+    free(kp);
+    return LCKV_ORACLE_OK;
 }

@@ -50,6 +50,11 @@ def lib():
                                                     i32p, C.c_int, C.c_int, C.c_int, C.c_int,
                                                     C.c_int64, C.c_int, C.c_double, C.c_int, pp]
         L.lckv_oracle_prefill_iteration.restype = C.c_int
+        f32p = C.POINTER(C.c_float)
+        f64p = C.POINTER(C.c_double)
+        L.lckv_oracle_project_kv.argtypes = [u16p, u16p, u16p, f32p, f32p, C.c_int, i32p, C.c_int,
+                                             C.c_int, C.c_int, C.c_int, u16p, u16p, f64p, f64p]
+        L.lckv_oracle_project_kv.restype = C.c_int
         L.lckv_oracle_num_threads.restype = C.c_int
         _LIB = L
     return _LIB
@@ -219,3 +224,32 @@ def prefill_iteration(L, w, q_layers, k_layers, v_layers, K_slots, V_slots, lens
                                              float(scale), int(always_sink), _ptr_array(outs))
     _chk(rc, "prefill_iteration")
     return outs
+
+
+def project_kv(x, w_k, w_v, lens, n_kv_heads, head_dim, rope_cos=None, rope_sin=None):
+    """Keys and values of the new token from hidden states: x [B, d_model], w_k / w_v
+    [H_kv*d, d_model] (bf16 bits); optional rotary tables [n_pos, d/2] float32 applied to the key at
+    position lens[b].  Returns (k_bits, v_bits [B, H_kv, d] uint16, k_f64, v_f64 the unrounded values)."""
+    x, w_k, w_v = _u16(x), _u16(w_k), _u16(w_v)
+    lens = np.ascontiguousarray(lens, np.int32)
+    B, d_model = x.shape
+    F = n_kv_heads * head_dim
+    assert w_k.shape == (F, d_model) and w_v.shape == (F, d_model)
+    k_bits = np.empty((B, n_kv_heads, head_dim), np.uint16)
+    v_bits = np.empty_like(k_bits)
+    k_f = np.empty((B, n_kv_heads, head_dim), np.float64)
+    v_f = np.empty_like(k_f)
+    cp = sp = None
+    n_pos = 0
+    if rope_cos is not None:
+        rope_cos = np.ascontiguousarray(rope_cos, np.float32)
+        rope_sin = np.ascontiguousarray(rope_sin, np.float32)
+        assert rope_cos.shape == rope_sin.shape and rope_cos.shape[1] == head_dim // 2
+        n_pos = rope_cos.shape[0]
+        cp, sp = _p(rope_cos, C.c_float), _p(rope_sin, C.c_float)
+    rc = lib().lckv_oracle_project_kv(_p(x, C.c_uint16), _p(w_k, C.c_uint16), _p(w_v, C.c_uint16),
+                                      cp, sp, n_pos, _p(lens, C.c_int32), B, n_kv_heads, head_dim,
+                                      d_model, _p(k_bits, C.c_uint16), _p(v_bits, C.c_uint16),
+                                      _p(k_f, C.c_double), _p(v_f, C.c_double))
+    _chk(rc, "project_kv")
+    return k_bits, v_bits, k_f, v_f
