@@ -197,6 +197,37 @@ int lckv_append_kv(lckv_cache_t* cache, int32_t slot, const void* k_new, const v
                    int32_t batch, int32_t advance_len, void* stream);
 
 /*
+ * Produce-and-append (Section 2.1: W_K and W_V map a hidden representation to
+ * its key and value, and in the condensed model only the top layer and the
+ * warmup layers still have them): for every b < batch computes
+ *     k[b, f] = sum_c w_k[f, c] x[b, c],   v[b, f] = sum_c w_v[f, c] x[b, c]
+ * on the tensor cores (bf16 inputs, fp32 accumulation, one rounding to bf16)
+ * and stores them as row len[b] of slot `slot` - lckv_append_kv without the
+ * round trip of k and v through device memory.
+ *   x        [batch, d_model] bf16, device, 16-byte aligned, row-major
+ *   w_k, w_v [H_kv * d_h, d_model] bf16, device, 16-byte aligned, row-major
+ *            (row f = output feature = kv head f / d_h, dimension f % d_h)
+ *   rope_cos, rope_sin  both NULL, or [rope_positions, d_h / 2] fp32 device
+ *            tables: the key (never the value) is then rotated by the token's
+ *            position p = len[b] in the half-split pairing
+ *              k'[i]         = k[i] cos[p,i] - k[i + d_h/2] sin[p,i]
+ *              k'[i + d_h/2] = k[i + d_h/2] cos[p,i] + k[i] sin[p,i],  i < d_h/2
+ *            (rotary position embedding as Llama models apply it; the paper
+ *            does not restate it, so it is optional and the tables - hence the
+ *            frequencies - are the caller's).
+ *   advance_len as in lckv_append_kv.
+ * Requirements: d_model a multiple of 64, H_kv * d_h a multiple of 128.
+ * Errors: EINVAL (null / misaligned pointer, bad shape, one table without the
+ * other, rope_positions <= some len[b]), ECAPACITY as lckv_append_kv, ECUDA.
+ * A device-side wait that runs out shows in lckv_cache_status (LCKV_ETIMEOUT).
+ * The library keeps descriptors of x, w_k, w_v keyed by address and shape.
+ */
+int lckv_project_append_kv(lckv_cache_t* cache, int32_t slot, const void* x, int32_t d_model,
+                           const void* w_k, const void* w_v, const float* rope_cos,
+                           const float* rope_sin, int32_t rope_positions, int32_t batch,
+                           int32_t advance_len, void* stream);
+
+/*
  * Decode attention of one layer for one new token per sequence (Section 2.1):
  *   out[b,h] = sum_j softmax_j( scale * <q[b,h], K[b,kv(h),j]> ) * V[b,kv(h),j]
  * over the visible rows j of slot `slot`: j < len[b] (LCKV_MODE_CONDENSED,

@@ -46,6 +46,7 @@ SIGNATURES = {
     "lckv_cache_slot_ptrs": (C.c_int, [_vp, _i32, _vpp, _vpp]),
     "lckv_cache_page_table": (C.c_int, [_vp, _i32p, _i32p]),
     "lckv_append_kv": (C.c_int, [_vp, _i32, _vp, _vp, _i32, _i32, _vp]),
+    "lckv_project_append_kv": (C.c_int, [_vp, _i32, _vp, _i32, _vp, _vp, _vp, _vp, _i32, _i32, _i32, _vp]),
     "lckv_decode_attention": (C.c_int, [_vp, _i32, _i32, _vp, _vp, _vp, _i32, _vp]),
     "lckv_layer_stack_step": (C.c_int, [_vp, _vpp, _vpp, _vpp, _vpp, _i32, _vp]),
     "lckv_layer_stack_step_host": (C.c_int, [_vp, _vpp, _vpp, _vpp, _vpp, _i32, _vp]),
@@ -229,6 +230,16 @@ class Cache:
         batch = k_new.shape[0] if batch is None else batch
         _chk(lib().lckv_append_kv(self.h, slot, _ptr(k_new), _ptr(v_new), batch, advance_len,
                                   _stream(stream)), "lckv_append_kv")
+
+    def lckv_project_append_kv(self, slot, x, w_k, w_v, rope_cos=None, rope_sin=None, batch=None,
+                               advance_len=0, stream=None):
+        """x [batch, d_model], w_k / w_v [H_kv*d_h, d_model] bf16 device tensors; optional rotary
+        tables [positions, d_h/2] fp32."""
+        batch = x.shape[0] if batch is None else batch
+        n_pos = 0 if rope_cos is None else rope_cos.shape[0]
+        _chk(lib().lckv_project_append_kv(self.h, slot, _ptr(x), x.shape[1], _ptr(w_k), _ptr(w_v),
+                                          _ptr(rope_cos), _ptr(rope_sin), n_pos, batch, advance_len,
+                                          _stream(stream)), "lckv_project_append_kv")
 
     def lckv_decode_attention(self, slot, mode, q, out=None, lse=None, batch=None, stream=None):
         batch = q.shape[0] if batch is None else batch

@@ -11,6 +11,7 @@
 #include "../../include/lckv.h"
 #include "lckv_attn_alu.cuh"
 #include "lckv_attn_mma.cuh"
+#include "lckv_project.cuh"
 #include "lckv_prefill.cuh"
 #include "lckv_prefill_tc5.cuh"
 #include "lckv_small_kernels.cuh"
@@ -107,6 +108,9 @@ struct lckv_cache {
     // CUDA graph of one step, valid for the argument pointers it was captured with
     cudaGraphExec_t graph_exec;
     std::vector<const void*> graph_key;
+    // descriptors of the producer's operands (x, W_K, W_V), keyed by address and shape
+    struct OperandMap { const void* ptr; uint64_t rows, cols; int box_rows; CUtensorMap tm; };
+    std::vector<OperandMap> operand_maps;
 };
 
 namespace {
@@ -790,6 +794,9 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
               cuda_ok(cudaFuncSetAttribute(lckv::attn_mma_kernel<64, true>,
                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            lckv::kMmaSmemBytes)) &&
+              cuda_ok(cudaFuncSetAttribute(lckv::project_kv_kernel,
+                                           cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                           lckv::proj_smem_bytes(256, 4))) &&
               cuda_ok(cudaFuncSetAttribute(lckv::prefill_tc5_kernel<128>,
                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            lckv::tc5_smem_bytes<128>())) &&
@@ -914,6 +921,87 @@ int lckv_append_kv(lckv_cache_t* c, int32_t slot, const void* k_new, const void*
     if (int rc = ensure_pages(c, batch, 1)) return rc;
     if (int rc = sync_page_table(c, st)) return rc;
     if (int rc = launch_append(c, slot, k_new, v_new, batch, st)) return rc;
+    if (advance_len) {
+        if (int rc = launch_advance(c, batch, st)) return rc;
+        mirror_advance(c, batch);
+    }
+    return LCKV_OK;
+}
+
+namespace {
+
+// Tensor map of a row-major bf16 matrix [rows, cols] with boxes of box_rows x 64 columns; kept per
+// (address, shape, box) so that repeated calls with the same weights do not re-encode.
+int operand_map(lckv_cache* c, const void* ptr, uint64_t rows, uint64_t cols, int box_rows,
+                CUtensorMap* out)
+{
+    for (const auto& m : c->operand_maps)
+        if (m.ptr == ptr && m.rows == rows && m.cols == cols && m.box_rows == box_rows) {
+            *out = m.tm;
+            return LCKV_OK;
+        }
+    if (c->operand_maps.size() >= 256) c->operand_maps.clear();
+    lckv_cache::OperandMap m;
+    m.ptr = ptr; m.rows = rows; m.cols = cols; m.box_rows = box_rows;
+    if (int rc = make_tensor_map_pitch(&m.tm, const_cast<void*>(ptr), rows, cols, cols * 2, box_rows))
+        return rc;
+    c->operand_maps.push_back(m);
+    *out = m.tm;
+    return LCKV_OK;
+}
+
+}  // namespace
+
+int lckv_project_append_kv(lckv_cache_t* c, int32_t slot, const void* x, int32_t d_model,
+                           const void* w_k, const void* w_v, const float* rope_cos,
+                           const float* rope_sin, int32_t rope_positions, int32_t batch,
+                           int32_t advance_len, void* stream)
+{
+    if (!c || !x || !w_k || !w_v || batch < 1 || batch > c->cfg.max_batch) return LCKV_EINVAL;
+    if (slot < 0 || slot >= c->plan.n_slots) return LCKV_EINVAL;
+    const int D = c->cfg.head_dim, F = c->cfg.n_kv_heads * D;
+    if (d_model < 64 || d_model % 64 || F % lckv::kProjBM) return LCKV_EINVAL;
+    if (((uintptr_t)x | (uintptr_t)w_k | (uintptr_t)w_v) & 15) return LCKV_EINVAL;
+    if ((rope_cos == nullptr) != (rope_sin == nullptr)) return LCKV_EINVAL;
+    if (rope_cos && (rope_positions < 1 || max_len(c, batch) >= rope_positions)) return LCKV_EINVAL;
+    if (max_len(c, batch) + 1 > c->cfg.max_seq) return LCKV_ECAPACITY;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (int rc = ensure_pages(c, batch, 1)) return rc;
+    if (int rc = sync_page_table(c, st)) return rc;
+
+    int NB = 16;
+    while (NB < batch && NB < 256) NB *= 2;
+    int n_stages = (192 * 1024) / lckv::proj_stage_bytes(NB);
+    if (n_stages > 8) n_stages = 8;
+    CUtensorMap tx, tk, tv;
+    if (int rc = operand_map(c, x, (uint64_t)batch, (uint64_t)d_model, NB, &tx)) return rc;
+    if (int rc = operand_map(c, w_k, (uint64_t)F, (uint64_t)d_model, lckv::kProjBM, &tk)) return rc;
+    if (int rc = operand_map(c, w_v, (uint64_t)F, (uint64_t)d_model, lckv::kProjBM, &tv)) return rc;
+
+    lckv::ProjParams p;
+    p.K = slot_k(c, slot);
+    p.V = slot_v(c, slot);
+    p.lens = c->d_lens;
+    p.rope_cos = rope_cos;
+    p.rope_sin = rope_sin;
+    p.status = c->d_status;
+    p.page_table = c->d_pt;
+    p.T_cap = c->cfg.max_seq;
+    p.pt_stride = c->pt_stride;
+    p.page_shift = c->page_shift;
+    p.B = batch;
+    p.H_kv = c->cfg.n_kv_heads;
+    p.D = D;
+    p.d_model = d_model;
+    p.NB = NB;
+    p.n_stages = n_stages;
+    p.n_sink = c->cfg.stream_sink;
+    p.k_tiles = F / lckv::kProjBM;
+    p.rope_positions = rope_positions;
+    const dim3 grid(2 * p.k_tiles, (batch + NB - 1) / NB);
+    lckv::project_kv_kernel<<<grid, lckv::kProjThreads, lckv::proj_smem_bytes(NB, n_stages), st>>>(
+        p, tx, tk, tv);
+    if (!cuda_ok(cudaGetLastError())) return LCKV_ECUDA;
     if (advance_len) {
         if (int rc = launch_advance(c, batch, st)) return rc;
         mirror_advance(c, batch);

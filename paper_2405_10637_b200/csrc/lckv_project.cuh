@@ -1,0 +1,213 @@
+// Fused K/V producer: k = x W_K^T, v = x W_V^T for the new token of every sequence, written
+// straight into row len[b] of a cache slot (paper Section 2.1: only the layers that own a cache
+// still compute K and V; W_K, W_V are the maps from hidden states to keys and values).
+//
+// The contraction runs on the 5th-generation tensor cores with the operands swapped, so that the
+// 128 rows of the MMA tile are output features (one head at d_h = 128, two at d_h = 64) and the
+// batch is the N side (16 ... 256): small decode batches do not pad a 128-row tile.
+//
+//   D^T [128 features x NB sequences] = W [128 x d_model] . x^T [d_model x NB]
+//
+//   warp 0     producer: 2-D TMA loads of the W tile [128 x 64] and the x tile [NB x 64] per k-step
+//   warp 1     one thread issues tcgen05.mma (both operands K-major in shared memory, fp32
+//              accumulator in tensor memory); tcgen05.commit frees the stage / signals the end
+//   warps 2-5  epilogue: tensor memory -> fp32 staging in shared memory (the pipeline's stages,
+//              idle by then), optional rotation of the key by its position (half-split pairs
+//              d, d + d_h/2 with caller-provided cos / sin tables), one rounding to bf16,
+//              16-byte stores into the cache row (ring position and page look-up as in
+//              append_kernel).
+//
+// Every wait is bounded; a wait that runs out sets the status word and the kernel returns.
+#pragma once
+#include "lckv_prefill_tc5.cuh"
+
+namespace lckv {
+
+constexpr int kProjThreads = 192;
+constexpr int kProjBM = 128;            // output features per CTA
+constexpr int kProjBK = 64;             // d_model columns per k-step (one 128-byte swizzled row)
+constexpr int kProjWBytes = kProjBM * 128;
+constexpr int kProjPad = 4;             // fp32 padding of a staged column (keeps 16-byte alignment)
+constexpr uint32_t kProjWaitLimit = 1u << 16;
+
+struct ProjParams {
+    uint16_t* K;              // slot's K and V tensors (contiguous or paged pool)
+    uint16_t* V;
+    const int32_t* lens;      // [B] tokens cached so far = position of the new token
+    const float* rope_cos;    // [rope_positions, D/2] or null
+    const float* rope_sin;
+    int32_t* status;
+    const int32_t* page_table;
+    int64_t T_cap;
+    int32_t pt_stride, page_shift;
+    int32_t B, H_kv, D, d_model;
+    int32_t NB;               // batch tile = N of the MMA (16, 32, 64, 128, 256)
+    int32_t n_stages;
+    int32_t n_sink;
+    int32_t k_tiles;          // feature tiles of K; tiles k_tiles .. 2*k_tiles-1 belong to V
+    int32_t rope_positions;
+};
+
+__host__ __device__ inline int proj_stage_bytes(int NB) { return kProjWBytes + NB * 128; }
+__host__ __device__ inline int proj_smem_bytes(int NB, int n_stages)
+{
+    const int pipe = n_stages * proj_stage_bytes(NB);
+    const int stage_out = NB * (kProjBM + kProjPad) * 4;
+    return (pipe > stage_out ? pipe : stage_out) + 256 + 1024;
+}
+
+__device__ __forceinline__ void bar_sync_epilogue()
+{
+    asm volatile("bar.sync 1, 128;" ::: "memory");
+}
+
+__global__ void __launch_bounds__(kProjThreads)
+project_kv_kernel(const ProjParams p, const __grid_constant__ CUtensorMap tmX,
+                  const __grid_constant__ CUtensorMap tmWk, const __grid_constant__ CUtensorMap tmWv)
+{
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int NB = p.NB, NS = p.n_stages;
+    const int stage_bytes = proj_stage_bytes(NB);
+    const int pipe = NS * stage_bytes;
+    const int stage_out = NB * (kProjBM + kProjPad) * 4;
+    const uint32_t bars = smem0 + (uint32_t)(pipe > stage_out ? pipe : stage_out);
+    // barriers: full[s] at bars + 8 s, empty[s] at bars + 64 + 8 s (s < 8), accumulator at +128
+    const uint32_t bFull = bars, bEmpty = bars + 64, bAcc = bars + 128, sTaddr = bars + 136;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    const int mt = blockIdx.x;                 // feature tile
+    const int b0 = blockIdx.y * NB;            // first sequence of the batch tile
+    const bool is_v = mt >= p.k_tiles;
+    const int f0 = (is_v ? mt - p.k_tiles : mt) * kProjBM;   // first feature within K or V
+    const int n_k = p.d_model / kProjBK;
+    const uint32_t tm_cols = NB < 32 ? 32u : (uint32_t)NB;
+
+    if (tid == 0) {
+        for (int s = 0; s < NS; ++s) { mbar_init(bFull + 8 * s, 1); mbar_init(bEmpty + 8 * s, 1); }
+        mbar_init(bAcc, 1);
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc(sTaddr, tm_cols);
+    tc5_fence_before();
+    __syncthreads();
+    tc5_fence_after();
+    uint32_t tmem_base;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(tmem_base) : "r"(sTaddr));
+
+    bool ok = true;
+    if (warp == 0) {
+        // ------------------------------------------------------------------ producer
+        if (lane == 0) {
+            const void* tmW = is_v ? (const void*)&tmWv : (const void*)&tmWk;
+            for (int k = 0; k < n_k && ok; ++k) {
+                const int s = k % NS;
+                if (k >= NS) ok = mbar_wait_bounded(bEmpty + 8 * s, ((k / NS) - 1) & 1, kProjWaitLimit);
+                if (!ok) break;
+                const uint32_t dst = smem0 + s * stage_bytes;
+                mbar_expect_tx(bFull + 8 * s, (uint32_t)stage_bytes);
+                tma_load_2d(dst, tmW, k * kProjBK, f0, bFull + 8 * s);
+                tma_load_2d(dst + kProjWBytes, &tmX, k * kProjBK, b0, bFull + 8 * s);
+            }
+            if (!ok) atomicExch(p.status, kStatusTimeout);
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            const uint32_t idesc = tc5_idesc(kProjBM, NB, 0);
+            for (int k = 0; k < n_k && ok; ++k) {
+                const int s = k % NS;
+                ok = mbar_wait_bounded(bFull + 8 * s, (k / NS) & 1, kProjWaitLimit);
+                if (!ok) break;
+                tc5_fence_after();
+                const uint32_t a0 = smem0 + s * stage_bytes, x0 = a0 + kProjWBytes;
+#pragma unroll
+                for (int ks = 0; ks < kProjBK / 16; ++ks)
+                    tc5_mma(tmem_base, tc5_desc(a0 + ks * 32, 16, 1024), tc5_desc(x0 + ks * 32, 16, 1024),
+                            idesc, (k > 0 || ks > 0));
+                tc5_commit(bEmpty + 8 * s);
+            }
+            if (ok) tc5_commit(bAcc);
+            else atomicExch(p.status, kStatusTimeout);
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue
+        const int q4 = warp & 3;
+        const int r = q4 * 32 + lane;                       // feature row of the tile = TMEM lane
+        const uint32_t lane_sel = (uint32_t)(q4 * 32) << 16;
+        const int et = tid - 64;                            // 0..127
+        const int ld = kProjBM + kProjPad;
+        ok = mbar_wait_bounded(bAcc, 0, kProjWaitLimit);
+        ok = __all_sync(0xffffffffu, ok);
+        if (ok) {
+            tc5_fence_after();
+            // accumulator -> staging [col][feature] fp32 (all MMAs are done: the stages are free)
+            for (int c0 = 0; c0 < NB; c0 += 32) {
+                uint32_t v[32];
+                // NB = 16: the allocation still has 32 columns; the upper 16 are read and dropped
+                tmem_ld32(tmem_base + lane_sel + c0, v);
+                const int nc = NB - c0 < 32 ? NB - c0 : 32;
+#pragma unroll
+                for (int c = 0; c < 32; ++c)
+                    if (c < nc)
+                        asm volatile("st.shared.b32 [%0], %1;" ::"r"(smem0 + (uint32_t)(((c0 + c) * ld + r) * 4)),
+                                     "r"(v[c]) : "memory");
+            }
+        } else if (lane == 0) {
+            atomicExch(p.status, kStatusTimeout);
+        }
+        bar_sync_epilogue();   // reached by all 128 epilogue threads, whatever the waits returned
+        // The accumulator barrier completes for all four warps or for none, so a warp that got
+        // here with ok set reads staging that the other three have written.
+        if (ok) {
+            const float* stg = reinterpret_cast<const float*>(smem_raw + (smem0 - smem_u32(smem_raw)));
+            const int D = p.D, half = D >> 1;
+            const int chunk = et & 15;                 // 8 features
+            const int fl = chunk * 8;                  // feature within the tile
+            const int feat = f0 + fl;                  // feature within K or V
+            const int kvh = feat / D, d = feat - kvh * D;
+            const bool rot = (!is_v) && p.rope_cos != nullptr;
+            const int fl_partner = d < half ? fl + half : fl - half;
+            uint16_t* base = is_v ? p.V : p.K;
+            for (int col = et >> 4; col < NB; col += 8) {
+                const int b = b0 + col;
+                if (b >= p.B) break;
+                const int32_t t = __ldg(p.lens + b);
+                int64_t row = t;
+                if (p.n_sink > 0 && row >= p.T_cap) row = p.n_sink + (row - p.n_sink) % (p.T_cap - p.n_sink);
+                if (row < 0 || row >= p.T_cap) continue;   // the host refuses such calls
+                int64_t dst_row = ((int64_t)b * p.H_kv + kvh) * p.T_cap + row;
+                if (p.page_table) {
+                    const int64_t id = __ldg(p.page_table + (int64_t)b * p.pt_stride + (row >> p.page_shift));
+                    dst_row = ((id * p.H_kv + kvh) << p.page_shift) + (row & ((1 << p.page_shift) - 1));
+                }
+                float x[8];
+                {
+                    const float4 lo = *reinterpret_cast<const float4*>(stg + col * ld + fl);
+                    const float4 hi = *reinterpret_cast<const float4*>(stg + col * ld + fl + 4);
+                    x[0] = lo.x; x[1] = lo.y; x[2] = lo.z; x[3] = lo.w;
+                    x[4] = hi.x; x[5] = hi.y; x[6] = hi.z; x[7] = hi.w;
+                }
+                if (rot) {
+                    const float* xp = stg + col * ld + fl_partner;
+                    const int pos = t < p.rope_positions ? t : p.rope_positions - 1;  // host checks the range
+                    const int i0 = d < half ? d : d - half;
+                    const float* cs = p.rope_cos + (size_t)pos * half + i0;
+                    const float* sn = p.rope_sin + (size_t)pos * half + i0;
+                    const float sgn = d < half ? -1.f : 1.f;
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        x[i] = fmaf(sgn * xp[i], __ldg(sn + i), x[i] * __ldg(cs + i));
+                }
+                const uint4 packed = make_uint4(cvt_bf16x2(x[0], x[1]), cvt_bf16x2(x[2], x[3]),
+                                                cvt_bf16x2(x[4], x[5]), cvt_bf16x2(x[6], x[7]));
+                *reinterpret_cast<uint4*>(base + dst_row * D + d) = packed;
+            }
+        }
+    }
+
+    tc5_fence_before();
+    __syncthreads();
+    if (warp == 0) tmem_dealloc(tmem_base, tm_cols);
+}
+
+}  // namespace lckv
