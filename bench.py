@@ -479,6 +479,79 @@ def run_prefill(args):
     cache.close()
 
 
+def run_project(args):
+    """--project D: times the fused key/value producer (x W_K^T, x W_V^T -> cache rows) for hidden width
+    D at the workload's head layout.  Several weight sets are used in turn so that their bytes exceed
+    the L2 (as the layers of a model would).  A side measurement, not the headline metric."""
+    from paper_2405_10637_b200 import binding as lk
+    wl, p = workload_params(args)
+    dm = args.project
+    B = args.batch or 64
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    F = wl.n_kv_heads * wl.head_dim
+    T_cap = 64
+    cfg = lk.make_config(2, 0, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, B, T_cap)
+    cache = lk.Cache(cfg, device=dev)
+    cache.lckv_cache_reset([5] * B)
+    w_bytes = 2 * F * dm * 2
+    n_sets = max(2, int(300e6 // w_bytes) + 1)           # > 126 MB of L2 between two uses of a set
+    wk = [syn.randn_bf16((F, dm), 10 + 2 * i, device=dev, std=dm ** -0.5) for i in range(n_sets)]
+    wv = [syn.randn_bf16((F, dm), 11 + 2 * i, device=dev, std=dm ** -0.5) for i in range(n_sets)]
+    x = syn.randn_bf16((B, dm), 3, device=dev)
+    half = wl.head_dim // 2
+    ang = torch.arange(T_cap, device=dev, dtype=torch.float64)[:, None] * \
+        (10000.0 ** (-2.0 * torch.arange(half, device=dev, dtype=torch.float64) / wl.head_dim))[None, :]
+    cos, sin = torch.cos(ang).float().contiguous(), torch.sin(ang).float().contiguous()
+    stream = torch.cuda.current_stream()
+    it = [0]
+
+    def f():
+        i = it[0] % n_sets
+        it[0] += 1
+        cache.lckv_project_append_kv(0, x, wk[i], wv[i], cos, sin, advance_len=0)
+    for _ in range(max(3, args.warmup) + n_sets):
+        f()
+    torch.cuda.synchronize()
+    # One call is 10-50 us of device time, less than a Python call costs on the host: replay a captured
+    # graph of one call per weight set so that the events see the device, not the interpreter.
+    graph = torch.cuda.CUDAGraph()
+    side = torch.cuda.Stream()
+    side.wait_stream(stream)
+    with torch.cuda.graph(graph, stream=side):
+        for _ in range(n_sets):
+            f()
+    torch.cuda.synchronize()
+    for _ in range(3):
+        graph.replay()
+    torch.cuda.synchronize()
+    ms = time_steps(graph.replay, args.steps, stream) / (args.steps * n_sets)
+    assert cache.lckv_cache_status() == 0, "device-side wait timed out"
+    flops = 2.0 * B * 2 * F * dm
+    byts = w_bytes + B * dm * 2 + 2 * B * F * 2
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            pk = json.load(fh)
+            peak_tf, peak_gb, kind = float(pk["bf16_tflops"]), float(pk["hbm_gbs"]), "measured"
+    except Exception:
+        peak_tf, peak_gb, kind = 1590.0, 6650.0, "fallback"
+    tf = flops / (ms * 1e-3) / 1e12
+    gbs = byts / (ms * 1e-3) / 1e9
+    hbm_bound = byts / peak_gb / 1e9 >= flops / peak_tf / 1e12
+    roof = {"bound": "hbm", "achieved": gbs, "peak": peak_gb, "unit": "GB/s", "frac": gbs / peak_gb} if hbm_bound \
+        else {"bound": "tensor", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": tf / peak_tf}
+    roof.update({"traffic": None, "peak_kind": kind, "kernel": "project_kv_kernel", "tflops": tf, "GBps": gbs,
+                 "algorithmic_bytes_per_launch": byts, "us_per_launch": ms * 1e3})
+    print(json.dumps({
+        "metric": "key/value producer (projection + rotary + append) us per call", "value": ms * 1e3,
+        "unit": "us", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
+        "higher_is_better": False, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": f"{wl.name} head layout, d_model {dm}, B={B}, {n_sets} weight sets in turn",
+                   "l2": "weight sets in rotation exceed L2"},
+        "roofline": roof}))
+    cache.close()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -499,6 +572,8 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prefill", type=int, default=0,
                     help="N > 0: time the prompt-encoding attention on N-token prompts instead")
+    ap.add_argument("--project", type=int, default=0,
+                    help="D > 0: time the fused key/value producer for hidden width D instead")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
     if args.impl == "reference":
@@ -508,6 +583,8 @@ def main():
             raise SystemExit("bench.py needs a CUDA device (the CUDA library has no CPU fallback)")
         if args.prefill:
             run_prefill(args)
+        elif args.project:
+            run_project(args)
         else:
             run_ours(args)
 

@@ -998,10 +998,25 @@ int lckv_project_append_kv(lckv_cache_t* c, int32_t slot, const void* x, int32_t
     p.n_sink = c->cfg.stream_sink;
     p.k_tiles = F / lckv::kProjBM;
     p.rope_positions = rope_positions;
-    const dim3 grid(2 * p.k_tiles, (batch + NB - 1) / NB);
-    lckv::project_kv_kernel<<<grid, lckv::kProjThreads, lckv::proj_smem_bytes(NB, n_stages), st>>>(
-        p, tx, tk, tv);
-    if (!cuda_ok(cudaGetLastError())) return LCKV_ECUDA;
+    // Few feature tiles (small batch): split d_model over a cluster so that more SMs stream weights.
+    const int tiles = 2 * p.k_tiles * ((batch + NB - 1) / NB);
+    const int n_k = d_model / lckv::kProjBK;
+    int ks = 1;
+    while (ks < 8 && tiles * ks * 2 <= c->sm_count && n_k % (ks * 2) == 0 && n_k / (ks * 2) >= 4) ks *= 2;
+    p.k_split = ks;
+    cudaLaunchConfig_t lc = {};
+    lc.gridDim = dim3(2 * p.k_tiles, (batch + NB - 1) / NB, ks);
+    lc.blockDim = dim3(lckv::kProjThreads);
+    lc.dynamicSmemBytes = lckv::proj_smem_bytes(NB, n_stages);
+    lc.stream = st;
+    cudaLaunchAttribute at[1];
+    at[0].id = cudaLaunchAttributeClusterDimension;
+    at[0].val.clusterDim.x = 1;
+    at[0].val.clusterDim.y = 1;
+    at[0].val.clusterDim.z = ks;
+    lc.attrs = at;
+    lc.numAttrs = 1;
+    if (!cuda_ok(cudaLaunchKernelEx(&lc, lckv::project_kv_kernel, p, tx, tk, tv))) return LCKV_ECUDA;
     if (advance_len) {
         if (int rc = launch_advance(c, batch, st)) return rc;
         mirror_advance(c, batch);

@@ -17,6 +17,13 @@
 //              16-byte stores into the cache row (ring position and page look-up as in
 //              append_kernel).
 //
+// Small batches are bound by streaming the weights, and a layer has only (2 H_kv d_h / 128) feature
+// tiles - 64 at the 7B width, fewer than the SMs.  The launch may therefore split d_model over a
+// thread-block cluster of k_split CTAs (cluster dimension z): each CTA accumulates its share of the
+// k-steps, all write their fp32 tile to their own shared memory, and each CTA finishes a share of
+// the tile's columns, adding the other CTAs' partial values through distributed shared memory
+// (two cluster barriers: tiles written / tiles read).
+//
 // Every wait is bounded; a wait that runs out sets the status word and the kernel returns.
 #pragma once
 #include "lckv_prefill_tc5.cuh"
@@ -46,6 +53,7 @@ struct ProjParams {
     int32_t n_sink;
     int32_t k_tiles;          // feature tiles of K; tiles k_tiles .. 2*k_tiles-1 belong to V
     int32_t rope_positions;
+    int32_t k_split;          // CTAs of a cluster that share one tile's k-steps (1, 2, 4, 8)
 };
 
 __host__ __device__ inline int proj_stage_bytes(int NB) { return kProjWBytes + NB * 128; }
@@ -56,9 +64,30 @@ __host__ __device__ inline int proj_smem_bytes(int NB, int n_stages)
     return (pipe > stage_out ? pipe : stage_out) + 256 + 1024;
 }
 
-__device__ __forceinline__ void bar_sync_epilogue()
+__device__ __forceinline__ uint32_t cluster_ctarank()
 {
-    asm volatile("bar.sync 1, 128;" ::: "memory");
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// Hardware barrier over all threads of the cluster (every thread of every CTA executes it).
+__device__ __forceinline__ void cluster_sync_all()
+{
+    __syncwarp();
+    asm volatile("barrier.cluster.arrive.release;" ::: "memory");
+    asm volatile("barrier.cluster.wait.acquire;" ::: "memory");
+}
+// 16 bytes of another CTA's shared memory: `addr` is the address in this CTA's own window.
+__device__ __forceinline__ float4 ld_cluster_f4(uint32_t addr, uint32_t rank)
+{
+    uint32_t ra;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(ra) : "r"(addr), "r"(rank));
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0,%1,%2,%3}, [%4];"
+                 : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w)
+                 : "r"(ra)
+                 : "memory");
+    return v;
 }
 
 __global__ void __launch_bounds__(kProjThreads)
@@ -79,7 +108,10 @@ project_kv_kernel(const ProjParams p, const __grid_constant__ CUtensorMap tmX,
     const int b0 = blockIdx.y * NB;            // first sequence of the batch tile
     const bool is_v = mt >= p.k_tiles;
     const int f0 = (is_v ? mt - p.k_tiles : mt) * kProjBM;   // first feature within K or V
-    const int n_k = p.d_model / kProjBK;
+    const int KS = p.k_split;
+    const uint32_t rank = KS > 1 ? cluster_ctarank() : 0u;
+    const int n_k = p.d_model / kProjBK / KS;       // this CTA's k-steps
+    const int k_first = (int)rank * n_k;
     const uint32_t tm_cols = NB < 32 ? 32u : (uint32_t)NB;
 
     if (tid == 0) {
@@ -105,8 +137,8 @@ project_kv_kernel(const ProjParams p, const __grid_constant__ CUtensorMap tmX,
                 if (!ok) break;
                 const uint32_t dst = smem0 + s * stage_bytes;
                 mbar_expect_tx(bFull + 8 * s, (uint32_t)stage_bytes);
-                tma_load_2d(dst, tmW, k * kProjBK, f0, bFull + 8 * s);
-                tma_load_2d(dst + kProjWBytes, &tmX, k * kProjBK, b0, bFull + 8 * s);
+                tma_load_2d(dst, tmW, (k_first + k) * kProjBK, f0, bFull + 8 * s);
+                tma_load_2d(dst + kProjWBytes, &tmX, (k_first + k) * kProjBK, b0, bFull + 8 * s);
             }
             if (!ok) atomicExch(p.status, kStatusTimeout);
         }
@@ -134,7 +166,6 @@ project_kv_kernel(const ProjParams p, const __grid_constant__ CUtensorMap tmX,
         const int q4 = warp & 3;
         const int r = q4 * 32 + lane;                       // feature row of the tile = TMEM lane
         const uint32_t lane_sel = (uint32_t)(q4 * 32) << 16;
-        const int et = tid - 64;                            // 0..127
         const int ld = kProjBM + kProjPad;
         ok = mbar_wait_bounded(bAcc, 0, kProjWaitLimit);
         ok = __all_sync(0xffffffffu, ok);
@@ -155,57 +186,76 @@ project_kv_kernel(const ProjParams p, const __grid_constant__ CUtensorMap tmX,
         } else if (lane == 0) {
             atomicExch(p.status, kStatusTimeout);
         }
-        bar_sync_epilogue();   // reached by all 128 epilogue threads, whatever the waits returned
-        // The accumulator barrier completes for all four warps or for none, so a warp that got
-        // here with ok set reads staging that the other three have written.
-        if (ok) {
-            const float* stg = reinterpret_cast<const float*>(smem_raw + (smem0 - smem_u32(smem_raw)));
-            const int D = p.D, half = D >> 1;
-            const int chunk = et & 15;                 // 8 features
-            const int fl = chunk * 8;                  // feature within the tile
-            const int feat = f0 + fl;                  // feature within K or V
-            const int kvh = feat / D, d = feat - kvh * D;
-            const bool rot = (!is_v) && p.rope_cos != nullptr;
-            const int fl_partner = d < half ? fl + half : fl - half;
-            uint16_t* base = is_v ? p.V : p.K;
-            for (int col = et >> 4; col < NB; col += 8) {
-                const int b = b0 + col;
-                if (b >= p.B) break;
-                const int32_t t = __ldg(p.lens + b);
-                int64_t row = t;
-                if (p.n_sink > 0 && row >= p.T_cap) row = p.n_sink + (row - p.n_sink) % (p.T_cap - p.n_sink);
-                if (row < 0 || row >= p.T_cap) continue;   // the host refuses such calls
-                int64_t dst_row = ((int64_t)b * p.H_kv + kvh) * p.T_cap + row;
-                if (p.page_table) {
-                    const int64_t id = __ldg(p.page_table + (int64_t)b * p.pt_stride + (row >> p.page_shift));
-                    dst_row = ((id * p.H_kv + kvh) << p.page_shift) + (row & ((1 << p.page_shift) - 1));
-                }
-                float x[8];
-                {
-                    const float4 lo = *reinterpret_cast<const float4*>(stg + col * ld + fl);
-                    const float4 hi = *reinterpret_cast<const float4*>(stg + col * ld + fl + 4);
-                    x[0] = lo.x; x[1] = lo.y; x[2] = lo.z; x[3] = lo.w;
-                    x[4] = hi.x; x[5] = hi.y; x[6] = hi.z; x[7] = hi.w;
-                }
-                if (rot) {
-                    const float* xp = stg + col * ld + fl_partner;
-                    const int pos = t < p.rope_positions ? t : p.rope_positions - 1;  // host checks the range
-                    const int i0 = d < half ? d : d - half;
-                    const float* cs = p.rope_cos + (size_t)pos * half + i0;
-                    const float* sn = p.rope_sin + (size_t)pos * half + i0;
-                    const float sgn = d < half ? -1.f : 1.f;
-#pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        x[i] = fmaf(sgn * xp[i], __ldg(sn + i), x[i] * __ldg(cs + i));
-                }
-                const uint4 packed = make_uint4(cvt_bf16x2(x[0], x[1]), cvt_bf16x2(x[2], x[3]),
-                                                cvt_bf16x2(x[4], x[5]), cvt_bf16x2(x[6], x[7]));
-                *reinterpret_cast<uint4*>(base + dst_row * D + d) = packed;
+    }
+
+    // All tiles of the cluster are in their CTAs' staging areas (or a wait ran out and the status
+    // word says so); every thread of every CTA reaches the barriers below.
+    tc5_fence_before();
+    __syncthreads();
+    if (KS > 1) cluster_sync_all();
+
+    if (warp >= 2 && ok) {
+        const int et = tid - 64;                            // 0..127
+        const int ld = kProjBM + kProjPad;
+        const float* stg = reinterpret_cast<const float*>(smem_raw + (smem0 - smem_u32(smem_raw)));
+        const int D = p.D, half = D >> 1;
+        const int chunk = et & 15;                 // 8 features
+        const int fl = chunk * 8;                  // feature within the tile
+        const int feat = f0 + fl;                  // feature within K or V
+        const int kvh = feat / D, d = feat - kvh * D;
+        const bool rot = (!is_v) && p.rope_cos != nullptr;
+        const int fl_partner = d < half ? fl + half : fl - half;
+        uint16_t* base = is_v ? p.V : p.K;
+        // the CTAs of a cluster share the columns: rank r finishes columns 8 r .. 8 r + 7 (mod 8 KS)
+        for (int col = (et >> 4) + 8 * (int)rank; col < NB; col += 8 * KS) {
+            const int b = b0 + col;
+            if (b >= p.B) break;
+            const int32_t t = __ldg(p.lens + b);
+            int64_t row = t;
+            if (p.n_sink > 0 && row >= p.T_cap) row = p.n_sink + (row - p.n_sink) % (p.T_cap - p.n_sink);
+            if (row < 0 || row >= p.T_cap) continue;   // the host refuses such calls
+            int64_t dst_row = ((int64_t)b * p.H_kv + kvh) * p.T_cap + row;
+            if (p.page_table) {
+                const int64_t id = __ldg(p.page_table + (int64_t)b * p.pt_stride + (row >> p.page_shift));
+                dst_row = ((id * p.H_kv + kvh) << p.page_shift) + (row & ((1 << p.page_shift) - 1));
             }
+            // this CTA's share plus the other ranks' (same offsets in their shared memory)
+            auto tile8 = [&](int f, float (&o)[8]) {
+                const float4 lo = *reinterpret_cast<const float4*>(stg + col * ld + f);
+                const float4 hi = *reinterpret_cast<const float4*>(stg + col * ld + f + 4);
+                o[0] = lo.x; o[1] = lo.y; o[2] = lo.z; o[3] = lo.w;
+                o[4] = hi.x; o[5] = hi.y; o[6] = hi.z; o[7] = hi.w;
+                for (int rk = 0; rk < KS; ++rk) {
+                    if (rk == (int)rank) continue;
+                    const uint32_t a = smem0 + (uint32_t)((col * ld + f) * 4);
+                    const float4 rl = ld_cluster_f4(a, (uint32_t)rk);
+                    const float4 rh = ld_cluster_f4(a + 16, (uint32_t)rk);
+                    o[0] += rl.x; o[1] += rl.y; o[2] += rl.z; o[3] += rl.w;
+                    o[4] += rh.x; o[5] += rh.y; o[6] += rh.z; o[7] += rh.w;
+                }
+            };
+            float x[8];
+            tile8(fl, x);
+            if (rot) {
+                float xp[8];
+                tile8(fl_partner, xp);
+                const int pos = t < p.rope_positions ? t : p.rope_positions - 1;  // host checks the range
+                const int i0 = d < half ? d : d - half;
+                const float* cs = p.rope_cos + (size_t)pos * half + i0;
+                const float* sn = p.rope_sin + (size_t)pos * half + i0;
+                const float sgn = d < half ? -1.f : 1.f;
+#pragma unroll
+                for (int i = 0; i < 8; ++i)
+                    x[i] = fmaf(sgn * xp[i], __ldg(sn + i), x[i] * __ldg(cs + i));
+            }
+            const uint4 packed = make_uint4(cvt_bf16x2(x[0], x[1]), cvt_bf16x2(x[2], x[3]),
+                                            cvt_bf16x2(x[4], x[5]), cvt_bf16x2(x[6], x[7]));
+            *reinterpret_cast<uint4*>(base + dst_row * D + d) = packed;
         }
     }
 
-    tc5_fence_before();
+    // a CTA's shared memory must outlive the other CTAs' reads
+    if (KS > 1) cluster_sync_all();
     __syncthreads();
     if (warp == 0) tmem_dealloc(tmem_base, tm_cols);
 }

@@ -123,6 +123,23 @@ def test_produced_rows_match_oracle(shape, B, rope):
     c.close()
 
 
+@pytest.mark.parametrize("rope", [False, True])
+@pytest.mark.parametrize("B", [3, 40, 300])
+@pytest.mark.parametrize("shape", ["d64_split4", "d128_split2", "d128_split8"])
+def test_hidden_width_split_over_a_cluster(shape, B, rope):
+    """Hidden widths with enough k-steps that the launch shares a tile among 2, 4 or 8 CTAs (their
+    partial tiles are added through distributed shared memory before the rows are stored)."""
+    kw = {"d64_split4": dict(Hq=4, Hkv=4, d=64), "d128_split2": dict(Hq=2, Hkv=2, d=128),
+          "d128_split8": dict(Hq=1, Hkv=1, d=128)}[shape]
+    d_model = {"d64_split4": 1024, "d128_split2": 512, "d128_split8": 2048}[shape]
+    T_cap = 12
+    lens = syn.ragged_lengths(B, 0, T_cap - 2, 177 + B).numpy()
+    c = Case(L=2, w=0, lens=lens, T_cap=T_cap, seed=9, poison=False, **kw)
+    produce(c, 0, d_model, rope, seed=2900 + B)
+    attend_and_compare(c, 0, seed=33)
+    c.close()
+
+
 def test_produce_into_warmup_slot_without_advancing():
     """A warmup layer's own cache (slot 1), lengths left alone (the step's other layers follow)."""
     lens = [3, 0, 9, 1]
