@@ -208,7 +208,7 @@ int lckv_append_kv(lckv_cache_t* cache, int32_t slot, const void* k_new, const v
  *   w_k, w_v [H_kv * d_h, d_model] bf16, device, 16-byte aligned, row-major
  *            (row f = output feature = kv head f / d_h, dimension f % d_h)
  *   rope_cos, rope_sin  both NULL, or [rope_positions, d_h / 2] fp32 device
- *            tables: the key (never the value) is then rotated by the token's
+ *            tables (16-byte aligned): the key (never the value) is then rotated by the token's
  *            position p = len[b] in the half-split pairing
  *              k'[i]         = k[i] cos[p,i] - k[i + d_h/2] sin[p,i]
  *              k'[i + d_h/2] = k[i + d_h/2] cos[p,i] + k[i] sin[p,i],  i < d_h/2

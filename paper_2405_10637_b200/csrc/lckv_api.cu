@@ -963,6 +963,7 @@ int lckv_project_append_kv(lckv_cache_t* c, int32_t slot, const void* x, int32_t
     if (d_model < 64 || d_model % 64 || F % lckv::kProjBM) return LCKV_EINVAL;
     if (((uintptr_t)x | (uintptr_t)w_k | (uintptr_t)w_v) & 15) return LCKV_EINVAL;
     if ((rope_cos == nullptr) != (rope_sin == nullptr)) return LCKV_EINVAL;
+    if (((uintptr_t)rope_cos | (uintptr_t)rope_sin) & 15) return LCKV_EINVAL;
     if (rope_cos && (rope_positions < 1 || max_len(c, batch) >= rope_positions)) return LCKV_EINVAL;
     if (max_len(c, batch) + 1 > c->cfg.max_seq) return LCKV_ECAPACITY;
     cudaStream_t st = static_cast<cudaStream_t>(stream);

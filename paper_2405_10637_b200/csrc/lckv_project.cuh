@@ -22,7 +22,7 @@
 // thread-block cluster of k_split CTAs (cluster dimension z): each CTA accumulates its share of the
 // k-steps, all write their fp32 tile to their own shared memory, and each CTA finishes a share of
 // the tile's columns, adding the other CTAs' partial values through distributed shared memory
-// (two cluster barriers: tiles written / tiles read).
+// (two cluster barriers: tiles written / tiles read).  The rotation tables must be 16-byte aligned.
 //
 // Every wait is bounded; a wait that runs out sets the status word and the kernel returns.
 #pragma once
@@ -194,63 +194,96 @@ project_kv_kernel(const ProjParams p, const __grid_constant__ CUtensorMap tmX,
     __syncthreads();
     if (KS > 1) cluster_sync_all();
 
-    if (warp >= 2 && ok) {
+    if (warp >= 2) {
         const int et = tid - 64;                            // 0..127
         const int ld = kProjBM + kProjPad;
-        const float* stg = reinterpret_cast<const float*>(smem_raw + (smem0 - smem_u32(smem_raw)));
-        const int D = p.D, half = D >> 1;
-        const int chunk = et & 15;                 // 8 features
-        const int fl = chunk * 8;                  // feature within the tile
-        const int feat = f0 + fl;                  // feature within K or V
-        const int kvh = feat / D, d = feat - kvh * D;
-        const bool rot = (!is_v) && p.rope_cos != nullptr;
-        const int fl_partner = d < half ? fl + half : fl - half;
-        uint16_t* base = is_v ? p.V : p.K;
-        // the CTAs of a cluster share the columns: rank r finishes columns 8 r .. 8 r + 7 (mod 8 KS)
-        for (int col = (et >> 4) + 8 * (int)rank; col < NB; col += 8 * KS) {
-            const int b = b0 + col;
-            if (b >= p.B) break;
-            const int32_t t = __ldg(p.lens + b);
-            int64_t row = t;
-            if (p.n_sink > 0 && row >= p.T_cap) row = p.n_sink + (row - p.n_sink) % (p.T_cap - p.n_sink);
-            if (row < 0 || row >= p.T_cap) continue;   // the host refuses such calls
-            int64_t dst_row = ((int64_t)b * p.H_kv + kvh) * p.T_cap + row;
-            if (p.page_table) {
-                const int64_t id = __ldg(p.page_table + (int64_t)b * p.pt_stride + (row >> p.page_shift));
-                dst_row = ((id * p.H_kv + kvh) << p.page_shift) + (row & ((1 << p.page_shift) - 1));
-            }
-            // this CTA's share plus the other ranks' (same offsets in their shared memory)
-            auto tile8 = [&](int f, float (&o)[8]) {
-                const float4 lo = *reinterpret_cast<const float4*>(stg + col * ld + f);
-                const float4 hi = *reinterpret_cast<const float4*>(stg + col * ld + f + 4);
-                o[0] = lo.x; o[1] = lo.y; o[2] = lo.z; o[3] = lo.w;
-                o[4] = hi.x; o[5] = hi.y; o[6] = hi.z; o[7] = hi.w;
+        float* stg = reinterpret_cast<float*>(smem_raw + (smem0 - smem_u32(smem_raw)));
+        // The CTAs of a cluster share the columns: rank r finishes columns [c_lo, c_hi).
+        const int per = NB / KS;
+        const int c_lo = (int)rank * per, c_hi = c_lo + per;
+        if (ok && KS > 1) {
+            // Pass 1: add the other CTAs' partial values of these columns into this CTA's staging
+            // (independent 16-byte loads through distributed shared memory, several in flight).
+            const int n4 = per * ld / 4;
+            float4* mine = reinterpret_cast<float4*>(stg + c_lo * ld);
+            const uint32_t a0 = smem0 + (uint32_t)(c_lo * ld * 4);
+            for (int i0 = et; i0 < n4; i0 += 128 * 4) {
+                float4 acc[4];
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = i0 + 128 * u;
+                    acc[u] = i < n4 ? mine[i] : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
                 for (int rk = 0; rk < KS; ++rk) {
                     if (rk == (int)rank) continue;
-                    const uint32_t a = smem0 + (uint32_t)((col * ld + f) * 4);
-                    const float4 rl = ld_cluster_f4(a, (uint32_t)rk);
-                    const float4 rh = ld_cluster_f4(a + 16, (uint32_t)rk);
-                    o[0] += rl.x; o[1] += rl.y; o[2] += rl.z; o[3] += rl.w;
-                    o[4] += rh.x; o[5] += rh.y; o[6] += rh.z; o[7] += rh.w;
-                }
-            };
-            float x[8];
-            tile8(fl, x);
-            if (rot) {
-                float xp[8];
-                tile8(fl_partner, xp);
-                const int pos = t < p.rope_positions ? t : p.rope_positions - 1;  // host checks the range
-                const int i0 = d < half ? d : d - half;
-                const float* cs = p.rope_cos + (size_t)pos * half + i0;
-                const float* sn = p.rope_sin + (size_t)pos * half + i0;
-                const float sgn = d < half ? -1.f : 1.f;
+                    float4 rv[4];
 #pragma unroll
-                for (int i = 0; i < 8; ++i)
-                    x[i] = fmaf(sgn * xp[i], __ldg(sn + i), x[i] * __ldg(cs + i));
+                    for (int u = 0; u < 4; ++u) {
+                        const int i = i0 + 128 * u;
+                        rv[u] = i < n4 ? ld_cluster_f4(a0 + (uint32_t)i * 16, (uint32_t)rk)
+                                       : make_float4(0.f, 0.f, 0.f, 0.f);
+                    }
+#pragma unroll
+                    for (int u = 0; u < 4; ++u) {
+                        acc[u].x += rv[u].x; acc[u].y += rv[u].y; acc[u].z += rv[u].z; acc[u].w += rv[u].w;
+                    }
+                }
+#pragma unroll
+                for (int u = 0; u < 4; ++u) {
+                    const int i = i0 + 128 * u;
+                    if (i < n4) mine[i] = acc[u];
+                }
             }
-            const uint4 packed = make_uint4(cvt_bf16x2(x[0], x[1]), cvt_bf16x2(x[2], x[3]),
-                                            cvt_bf16x2(x[4], x[5]), cvt_bf16x2(x[6], x[7]));
-            *reinterpret_cast<uint4*>(base + dst_row * D + d) = packed;
+        }
+        asm volatile("bar.sync 1, 128;" ::: "memory");   // all four epilogue warps, whatever ok says
+        if (ok) {
+            // Pass 2: rotation, rounding, stores - from this CTA's shared memory only.
+            const int D = p.D, half = D >> 1;
+            const int chunk = et & 15;                 // 8 features
+            const int fl = chunk * 8;                  // feature within the tile
+            const int feat = f0 + fl;                  // feature within K or V
+            const int kvh = feat / D, d = feat - kvh * D;
+            const bool rot = (!is_v) && p.rope_cos != nullptr;
+            const int fl_partner = d < half ? fl + half : fl - half;
+            const int i0 = d < half ? d : d - half;
+            const float sgn = d < half ? -1.f : 1.f;
+            uint16_t* base = is_v ? p.V : p.K;
+            for (int col = c_lo + (et >> 4); col < c_hi; col += 8) {
+                const int b = b0 + col;
+                if (b >= p.B) break;
+                const int32_t t = __ldg(p.lens + b);
+                int64_t row = t;
+                if (p.n_sink > 0 && row >= p.T_cap) row = p.n_sink + (row - p.n_sink) % (p.T_cap - p.n_sink);
+                if (row < 0 || row >= p.T_cap) continue;   // the host refuses such calls
+                int64_t dst_row = ((int64_t)b * p.H_kv + kvh) * p.T_cap + row;
+                if (p.page_table) {
+                    const int64_t id = __ldg(p.page_table + (int64_t)b * p.pt_stride + (row >> p.page_shift));
+                    dst_row = ((id * p.H_kv + kvh) << p.page_shift) + (row & ((1 << p.page_shift) - 1));
+                }
+                float x[8];
+                {
+                    const float4 lo = *reinterpret_cast<const float4*>(stg + col * ld + fl);
+                    const float4 hi = *reinterpret_cast<const float4*>(stg + col * ld + fl + 4);
+                    x[0] = lo.x; x[1] = lo.y; x[2] = lo.z; x[3] = lo.w;
+                    x[4] = hi.x; x[5] = hi.y; x[6] = hi.z; x[7] = hi.w;
+                }
+                if (rot) {
+                    const float4 pl = *reinterpret_cast<const float4*>(stg + col * ld + fl_partner);
+                    const float4 ph = *reinterpret_cast<const float4*>(stg + col * ld + fl_partner + 4);
+                    const float xp[8] = {pl.x, pl.y, pl.z, pl.w, ph.x, ph.y, ph.z, ph.w};
+                    const int pos = t < p.rope_positions ? t : p.rope_positions - 1;  // host checks the range
+                    const float4* cs4 = reinterpret_cast<const float4*>(p.rope_cos + (size_t)pos * half + i0);
+                    const float4* sn4 = reinterpret_cast<const float4*>(p.rope_sin + (size_t)pos * half + i0);
+                    const float4 c0 = __ldg(cs4), c1 = __ldg(cs4 + 1), s0 = __ldg(sn4), s1 = __ldg(sn4 + 1);
+                    const float cs[8] = {c0.x, c0.y, c0.z, c0.w, c1.x, c1.y, c1.z, c1.w};
+                    const float sn[8] = {s0.x, s0.y, s0.z, s0.w, s1.x, s1.y, s1.z, s1.w};
+#pragma unroll
+                    for (int i = 0; i < 8; ++i) x[i] = fmaf(sgn * xp[i], sn[i], x[i] * cs[i]);
+                }
+                const uint4 packed = make_uint4(cvt_bf16x2(x[0], x[1]), cvt_bf16x2(x[2], x[3]),
+                                                cvt_bf16x2(x[4], x[5]), cvt_bf16x2(x[6], x[7]));
+                *reinterpret_cast<uint4*>(base + dst_row * D + d) = packed;
+            }
         }
     }
 
