@@ -269,10 +269,15 @@ int lckv_layer_stack_step(lckv_cache_t* cache, const void* const* q_layers,
  * The same step for callers whose activations live in HOST memory (pinned for
  * real overlap): copies every layer's q (and the k,v of layers that have them)
  * host->device into the cache's staging area, runs the step, copies every
- * layer's output device->host.  All on `stream`, asynchronous; synchronise the
- * stream before reading the outputs.  Needs host_staging = 1 at alloc.  When the
- * layers' host buffers are contiguous in memory (one allocation sliced per
- * layer) each direction is a single pitched copy instead of one copy per layer.
+ * layer's output device->host.  Asynchronous: the step is ordered after the work
+ * already queued on `stream`, and `stream` ends up waiting for the last copy, so
+ * synchronise `stream` before reading the outputs.  The copies themselves run
+ * on two streams the cache creates on the first such call (no device memory is
+ * allocated): the layers are cut into up to 8 chunks, a chunk's layers start
+ * when its queries have arrived and its outputs leave while later chunks
+ * compute.  Needs host_staging = 1 at alloc.  When the layers' host buffers are
+ * contiguous in memory (one allocation sliced per layer) a chunk is a single
+ * pitched copy per direction instead of one copy per layer.
  * Array arguments are HOST arrays of L HOST pointers with the shapes above.
  */
 int lckv_layer_stack_step_host(lckv_cache_t* cache, const void* const* q_layers_host,

@@ -108,6 +108,9 @@ struct lckv_cache {
     // CUDA graph of one step, valid for the argument pointers it was captured with
     cudaGraphExec_t graph_exec;
     std::vector<const void*> graph_key;
+    // host-buffer step: copy streams and events (created on first use when cfg.host_staging)
+    cudaStream_t s_in = nullptr, s_out = nullptr;
+    std::vector<cudaEvent_t> ev;          // [0] step start, [1] k/v in, [2] all out, then per chunk in / done
     // descriptors of the producer's operands (x, W_K, W_V), keyed by address and shape
     struct OperandMap { const void* ptr; uint64_t rows, cols; int box_rows; CUtensorMap tm; };
     std::vector<OperandMap> operand_maps;
@@ -457,8 +460,14 @@ float step_keep_frac(const lckv_cache* c, int batch)
 }
 
 // The launches of one step, in the order the header states.
+// Events around layers of a step (host-buffer step: inputs arrive and outputs leave on other streams).
+struct StepHooks {
+    std::vector<cudaEvent_t> wait_before;   // per layer: wait for this event before the layer (or null)
+    std::vector<cudaEvent_t> record_after;  // per layer: record this event after the layer (or null)
+};
+
 int enqueue_step(lckv_cache* c, const void* const* q, void* const* out, const void* const* kn,
-                 const void* const* vn, int batch, cudaStream_t st)
+                 const void* const* vn, int batch, cudaStream_t st, const StepHooks* hooks = nullptr)
 {
     const Plan& pl = c->plan;
     const int L = c->cfg.n_layers;
@@ -473,6 +482,10 @@ int enqueue_step(lckv_cache* c, const void* const* q, void* const* out, const vo
     for (int l = 0; l < L; ++l) readers[pl.read_slot[l]] += 1;
     bool prev_attn = false;
     for (int l = 0; l < L; ++l) {
+        if (hooks && hooks->wait_before[l]) {
+            if (!cuda_ok(cudaStreamWaitEvent(st, hooks->wait_before[l], 0))) return LCKV_ECUDA;
+            prev_attn = false;   // the launch that follows an event wait waits in full
+        }
         if (pl.write_slot[l] >= 0 && pl.write_before[l]) {
             if (int rc = launch_append(c, pl.write_slot[l], kn[l], vn[l], batch, st)) return rc;
             prev_attn = false;
@@ -483,6 +496,10 @@ int enqueue_step(lckv_cache* c, const void* const* q, void* const* out, const vo
                                       st, early, keep))
             return rc;
         prev_attn = true;
+        if (hooks && hooks->record_after[l]) {
+            if (!cuda_ok(cudaEventRecord(hooks->record_after[l], st))) return LCKV_ECUDA;
+            prev_attn = false;
+        }
     }
     for (int l = 0; l < L; ++l)
         if (pl.write_slot[l] >= 0 && !pl.write_before[l])
@@ -832,6 +849,9 @@ int lckv_cache_free(lckv_cache_t* cache)
 {
     if (!cache) return LCKV_EINVAL;
     drop_graph(cache);
+    for (cudaEvent_t e : cache->ev) cudaEventDestroy(e);
+    if (cache->s_in) cudaStreamDestroy(cache->s_in);
+    if (cache->s_out) cudaStreamDestroy(cache->s_out);
     delete cache;
     return LCKV_OK;
 }
@@ -1089,16 +1109,61 @@ int lckv_layer_stack_step_host(lckv_cache_t* c, const void* const* q_host, void*
         }
     }
     uint8_t* skv = c->base + c->lay.off_stage_kv;
-    if (int rc = copy_layers(c->base + c->lay.off_stage_q, c->lay.stage_q_bytes, q_host, L, q_bytes, true, st))
-        return rc;
-    if (int rc = copy_layers(skv, 2 * c->lay.stage_kv_bytes, hk.data(), (int)hk.size(), kv_bytes, true, st))
+    // Copies run on two streams of the cache's own, so that the inputs of later layers arrive and
+    // the outputs of earlier layers leave while the layers in between compute.  The layers are cut
+    // into chunks; a chunk starts once its queries are on the device, and its outputs are fetched
+    // once it is done.  The caller's stream ends up waiting for the last copy.
+    const int n_chunks = L < 8 ? L : 8;
+    if (!c->s_in) {
+        if (!cuda_ok(cudaStreamCreateWithFlags(&c->s_in, cudaStreamNonBlocking)) ||
+            !cuda_ok(cudaStreamCreateWithFlags(&c->s_out, cudaStreamNonBlocking)))
+            return LCKV_ECUDA;
+    }
+    while ((int)c->ev.size() < 3 + 2 * n_chunks) {
+        cudaEvent_t e;
+        if (!cuda_ok(cudaEventCreateWithFlags(&e, cudaEventDisableTiming))) return LCKV_ECUDA;
+        c->ev.push_back(e);
+    }
+    cudaEvent_t ev_start = c->ev[0], ev_kv = c->ev[1], ev_out = c->ev[2];
+    // staging buffers are free once everything queued on the caller's stream so far has run
+    if (!cuda_ok(cudaEventRecord(ev_start, st)) || !cuda_ok(cudaStreamWaitEvent(c->s_in, ev_start, 0)))
+        return LCKV_ECUDA;
+    if (int rc = copy_layers(skv, 2 * c->lay.stage_kv_bytes, hk.data(), (int)hk.size(), kv_bytes, true, c->s_in))
         return rc;
     if (int rc = copy_layers(skv + c->lay.stage_kv_bytes, 2 * c->lay.stage_kv_bytes, hv.data(),
-                             (int)hv.size(), kv_bytes, true, st))
+                             (int)hv.size(), kv_bytes, true, c->s_in))
         return rc;
-    if (int rc = run_step(c, dq.data(), dout.data(), dk.data(), dv.data(), batch, st)) return rc;
-    return copy_layers(c->base + c->lay.off_stage_out, c->lay.stage_out_bytes,
-                       const_cast<const void* const*>(out_host), L, o_bytes, false, st);
+    if (!cuda_ok(cudaEventRecord(ev_kv, c->s_in)) || !cuda_ok(cudaStreamWaitEvent(st, ev_kv, 0)))
+        return LCKV_ECUDA;
+    StepHooks hooks;
+    hooks.wait_before.assign(L, nullptr);
+    hooks.record_after.assign(L, nullptr);
+    std::vector<int> first(n_chunks + 1);
+    for (int k = 0; k <= n_chunks; ++k) first[k] = (int)((int64_t)k * L / n_chunks);
+    for (int k = 0; k < n_chunks; ++k) {
+        const int l0 = first[k], n = first[k + 1] - l0;
+        if (int rc = copy_layers(c->base + c->lay.off_stage_q + (size_t)l0 * c->lay.stage_q_bytes,
+                                 c->lay.stage_q_bytes, q_host + l0, n, q_bytes, true, c->s_in))
+            return rc;
+        if (!cuda_ok(cudaEventRecord(c->ev[3 + 2 * k], c->s_in))) return LCKV_ECUDA;
+        hooks.wait_before[l0] = c->ev[3 + 2 * k];
+        hooks.record_after[l0 + n - 1] = c->ev[4 + 2 * k];
+    }
+    if (int rc = ensure_pages(c, batch, 1)) return rc;
+    if (int rc = sync_page_table(c, st)) return rc;
+    if (int rc = enqueue_step(c, dq.data(), dout.data(), dk.data(), dv.data(), batch, st, &hooks)) return rc;
+    mirror_advance(c, batch);
+    for (int k = 0; k < n_chunks; ++k) {
+        const int l0 = first[k], n = first[k + 1] - l0;
+        if (!cuda_ok(cudaStreamWaitEvent(c->s_out, c->ev[4 + 2 * k], 0))) return LCKV_ECUDA;
+        if (int rc = copy_layers(c->base + c->lay.off_stage_out + (size_t)l0 * c->lay.stage_out_bytes,
+                                 c->lay.stage_out_bytes, const_cast<const void* const*>(out_host) + l0, n,
+                                 o_bytes, false, c->s_out))
+            return rc;
+    }
+    if (!cuda_ok(cudaEventRecord(ev_out, c->s_out)) || !cuda_ok(cudaStreamWaitEvent(st, ev_out, 0)))
+        return LCKV_ECUDA;
+    return LCKV_OK;
 }
 
 int lckv_prefill_write_kv(lckv_cache_t* c, int32_t slot, const void* k, const void* v,
