@@ -169,6 +169,38 @@ def test_host_buffer_entry_point_matches():
     c.close()
 
 
+def test_host_buffer_steps_queued_back_to_back():
+    """More layers than copy chunks, mixed with device-buffer steps, and two host-buffer steps queued
+    without a synchronisation in between (the second step's input copies must not overtake the first
+    step's kernels, which still read the staging area)."""
+    c = Case(L=12, w=2, Hq=4, Hkv=2, d=64, lens=[7, 0, 130, 64], T_cap=160, seed=63, host_staging=1)
+    c.step(host=True)
+    c.step()
+    c.step(host=True, contiguous=True)
+    odt = torch.float32 if c.cfg.out_dtype else torch.bfloat16
+    queued = []
+    for _ in range(2):
+        q, kn, vn = c.step_inputs()
+        c.step_no += 1
+        qd = [t.pin_memory() for t in q]
+        knd = [None if t is None else t.pin_memory() for t in kn]
+        vnd = [None if t is None else t.pin_memory() for t in vn]
+        outs = [torch.empty((c.B, c.Hq, c.d), dtype=odt).pin_memory() for _ in range(c.L)]
+        c.cache.lckv_layer_stack_step_host(qd, outs, knd, vnd)
+        queued.append((q, kn, vn, outs, (qd, knd, vnd)))
+    torch.cuda.synchronize()
+    assert c.cache.lckv_cache_status() == 0
+    for q, kn, vn, outs, _ in queued:
+        want, _ = orc.stack_step(c.L, c.w, [syn.bits(t) for t in q],
+                                 [None if t is None else syn.bits(t) for t in kn],
+                                 [None if t is None else syn.bits(t) for t in vn],
+                                 c.hK, c.hV, c.lens, c.scale, top_variant=c.variant)
+        for l in range(c.L):
+            compare(outs[l], want[l], f"queued host step, layer {l}")
+    c.check_state()
+    c.close()
+
+
 def test_repeatable_bitwise():
     """Same inputs twice: identical bits (the merge order is fixed, not arrival order)."""
     outs = []
