@@ -17,7 +17,7 @@ from helpers import MAX_ABS, REL_L2
 pytestmark = pytest.mark.gpu
 
 
-def run_full(wl, B, lens, T_cap, n_samples, seed, top_variant=0, steps=1):
+def run_full(wl, B, lens, T_cap, n_samples, seed, top_variant=0, steps=1, check_at=None, fixed_inputs=False):
     L, Hq, Hkv, d = wl.n_layers, wl.n_q_heads, wl.n_kv_heads, wl.head_dim
     g = Hq // Hkv
     cfg = lk.make_config(L, wl.n_warmup, Hq, Hkv, d, B, T_cap, top_variant=top_variant)
@@ -32,12 +32,17 @@ def run_full(wl, B, lens, T_cap, n_samples, seed, top_variant=0, steps=1):
     rng = np.random.default_rng(seed)
     scale = d ** -0.5
     cur = lens.astype(np.int64).copy()
+    q = kv = outs = None
     for step in range(steps):
-        q = [syn.randn_bf16((B, Hq, d), 900 + l + 100 * step, device=dev, std=wl.std) for l in range(L)]
-        kv = [syn.randn_bf16((B, Hkv, d), 950 + l + 100 * step, device=dev, std=wl.std)
-              if plan["write_slot"][l] >= 0 else None for l in range(L)]
-        outs = [torch.full((B, Hq, d), float("nan"), dtype=torch.bfloat16, device=dev) for _ in range(L)]
+        if q is None or not fixed_inputs:
+            q = [syn.randn_bf16((B, Hq, d), 900 + l + 100 * step, device=dev, std=wl.std) for l in range(L)]
+            kv = [syn.randn_bf16((B, Hkv, d), 950 + l + 100 * step, device=dev, std=wl.std)
+                  if plan["write_slot"][l] >= 0 else None for l in range(L)]
+            outs = [torch.full((B, Hq, d), float("nan"), dtype=torch.bfloat16, device=dev) for _ in range(L)]
         cache.lckv_layer_stack_step(q, outs, kv, kv)
+        if check_at is not None and step not in check_at:
+            cur += 1
+            continue
         torch.cuda.synchronize()
         assert cache.lckv_cache_status() == 0
         for l in range(L):
@@ -65,6 +70,19 @@ def run_full(wl, B, lens, T_cap, n_samples, seed, top_variant=0, steps=1):
                 assert torch.equal(kt[b, :, row], kv[l][b]) and torch.equal(vt[b, :, row], kv[l][b])
         cur += 1
         assert cache.lckv_cache_lengths(B) == cur.tolist()
+    if fixed_inputs:
+        # every step appended the same k/v: the rows [len0, len0 + steps) of each fed slot must all
+        # hold them, bit for bit, and nothing beyond
+        torch.cuda.synchronize()
+        assert cache.lckv_cache_status() == 0
+        for l in range(L):
+            if plan["write_slot"][l] < 0:
+                continue
+            kt, vt = cache.slot_tensors(plan["write_slot"][l])
+            for b in rng.integers(B, size=min(B, 4)):
+                lo = int(lens[b])
+                want = kv[l][b][:, None, :].expand(-1, steps, -1)
+                assert torch.equal(kt[b, :, lo:lo + steps], want) and torch.equal(vt[b, :, lo:lo + steps], want)
     cache.close()
 
 
@@ -88,6 +106,24 @@ def test_tinyllama_batch_128_decode_steps():
     wl = syn.WORKLOADS["tinyllama"]
     lens = np.full(128, 512, np.int32)
     run_full(wl, 128, lens, 1536, n_samples=48, seed=3, steps=3)
+
+
+def test_tinyllama_1024_decode_steps_fill_the_cache():
+    """TinyLlama shape, B = 128, prompt 512 + 1024 generated tokens (the paper's 512+1024 setting): the
+    caches end exactly full; sampled rows are checked at the first steps, in the middle and at the end."""
+    wl = syn.WORKLOADS["tinyllama"]
+    lens = np.full(128, 512, np.int32)
+    run_full(wl, 128, lens, 1536, n_samples=24, seed=13, steps=1024, check_at={0, 1, 511, 1023},
+             fixed_inputs=True)
+
+
+def test_llama30b_2048_appends_small_batch():
+    """Llama-30B shape (60 layers, 52 heads), prompt 2048 + 2048 generated tokens at B = 2: every one
+    of the 2048 appended rows lands where it should."""
+    wl = syn.WORKLOADS["llama30b"]
+    lens = np.full(2, 2048, np.int32)
+    run_full(wl, 2, lens, 4096, n_samples=16, seed=14, steps=2048, check_at={0, 1024, 2047},
+             fixed_inputs=True)
 
 
 def test_llama30b_batch_256():
