@@ -12,6 +12,17 @@ from helpers import compare, NAN_BITS
 pytestmark = pytest.mark.gpu
 
 
+@pytest.fixture(params=["tc5", "mma"], autouse=True)
+def prefill_kernel(request, monkeypatch):
+    """Every test runs on both kernels of the operation: tcgen05 (the default) and mma.sync (the choice
+    is read when a cache is created)."""
+    if request.param == "tc5":
+        monkeypatch.delenv("LCKV_PREFILL_KERNEL", raising=False)
+    else:
+        monkeypatch.setenv("LCKV_PREFILL_KERNEL", request.param)
+    return request.param
+
+
 def make_cache(L, w, Hq, Hkv, d, lens, T_cap, out_dtype=0, variant=0, seed=0, std=1.0, poison=True):
     B = len(lens)
     cfg = lk.make_config(L, w, Hq, Hkv, d, B, T_cap, out_dtype=out_dtype, top_variant=variant)
@@ -163,11 +174,9 @@ def test_prefill_errors():
     c2.close()
 
 
-@pytest.mark.parametrize("kernel", ["tc5", "mma"])
-def test_prefill_on_paged_cache(kernel, monkeypatch):
-    """Prompt encoding over slots made of 64-row pages (scrambled page order), both kernels."""
+def test_prefill_on_paged_cache():
+    """Prompt encoding over slots made of 64-row pages (scrambled page order)."""
     from helpers import Case
-    monkeypatch.setenv("LCKV_PREFILL_KERNEL", kernel)
     lens = [130, 64, 1, 200, 65]
     c = Case(L=4, w=2, Hq=8, Hkv=2, d=64, lens=lens, T_cap=256, seed=17, std=0.5, page_rows=64, n_pages=14)
     dev, B, n_max = c.cache.device, len(lens), 200
