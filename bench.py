@@ -83,6 +83,8 @@ def workload_params(args):
         p = dict(batch=256, lo=3072, hi=3072, t_cap=3072, sweep=[256])
     elif args.workload == "sweep7b":
         p = dict(batch=64, lo=8192, hi=8192, t_cap=8192, sweep=[64])
+    elif args.workload == "gqa4":
+        p = dict(batch=256, lo=4096, hi=4096, t_cap=4096, sweep=[256])
     else:
         raise SystemExit(f"unknown workload {args.workload}")
     if args.batch:
@@ -280,7 +282,7 @@ def run_ours(args):
         grow = max(64, args.steps + args.warmup + 8)
         n_pages = int(1.02 * sum((int(x) + grow + args.page_rows - 1) // args.page_rows for x in lens)) + 8
     cfg = lk.make_config(L, wl.n_warmup, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, B, T_cap,
-                         host_staging=1, use_graph=1 if args.graph else 0,
+                         host_staging=1, use_graph=1 if args.graph else 0, kernel_kind=args.kernel_kind,
                          top_variant=args.top_variant, stream_sink=args.stream_sink,
                          page_rows=args.page_rows, n_pages=n_pages)
     cap = T_cap if args.stream_sink else 0
@@ -564,6 +566,8 @@ def main():
     ap.add_argument("--warmup-layers", type=int, default=None, help="override w")
     ap.add_argument("--top-variant", type=int, default=0)
     ap.add_argument("--graph", type=int, default=1)
+    ap.add_argument("--kernel-kind", type=int, default=0, choices=[0, 1],
+                    help="1: force the FP32-ALU attention kernel for grouped heads (0: automatic)")
     ap.add_argument("--page-rows", type=int, default=0,
                     help="P > 0: paged caches with P-row pages and a pool sized for the batch's lengths")
     ap.add_argument("--stream-sink", type=int, default=0,

@@ -83,8 +83,8 @@ typedef struct {
                               [B_max][ceil(T_cap / P)] serves every slot (all caches have the same
                               lengths).  Not combinable with stream_sink.                     */
     int32_t n_pages;       /* pool size per slot when page_rows > 0                            */
-    int32_t kernel_kind;   /* 0 = choose (tensor-core kernel when the query group is a dense
-                              MMA tile, else the FP32-ALU kernel); 1 = force FP32-ALU        */
+    int32_t kernel_kind;   /* 0 = choose (tensor-core kernel for query groups of 2 ... 7 and
+                              multiples of 8, else the FP32-ALU kernel); 1 = force FP32-ALU  */
 } lckv_config_t;
 
 /* Facts about a built cache that a caller or a benchmark may want. */

@@ -141,14 +141,24 @@ int validate_config(const lckv_config_t* c)
     return LCKV_OK;
 }
 
-// 1 = FP32-ALU kernel, 2 = tensor-core kernel (query groups that are multiples of 8).
+// 1 = FP32-ALU kernel, 2 = tensor-core kernel (query groups of 2 ... 7 and multiples of 8).
 int resolve_kernel_kind(const lckv_config_t& c)
 {
     const int g = c.n_q_heads / c.n_kv_heads;
     // the tensor-core kernel addresses cache rows through 32-bit TMA coordinates
     const uint64_t rows = c.page_rows ? (uint64_t)c.n_pages * c.n_kv_heads * (uint64_t)c.page_rows
                                       : (uint64_t)c.max_batch * c.n_kv_heads * (uint64_t)c.max_seq;
-    return (c.kernel_kind == 0 && g % 8 == 0 && rows < (1ull << 31)) ? 2 : 1;
+    // groups of 8 fill the N = 8 side of the MMA tile; smaller groups (2 ... 7) use it with the
+    // remaining columns zero, which still reads K and V once per group instead of once per head
+    const bool fits = g % 8 == 0 || (g >= 2 && g < 8);
+    return (c.kernel_kind == 0 && fits && rows < (1ull << 31)) ? 2 : 1;
+}
+
+// Query heads per pair of the tensor-core kernel: 8, or the whole group when it is smaller.
+int mma_heads_per_pair(const lckv_config_t& c)
+{
+    const int g = c.n_q_heads / c.n_kv_heads;
+    return g < 8 ? g : 8;
 }
 
 int workers_per_sm(const lckv_config_t& c)
@@ -398,9 +408,10 @@ int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out
     if (c->kernel_kind == 2) {
         lckv::MmaParams mp;
         mp.a = p;
-        mp.a.H_q = c->h_pairs;  // pairs per sequence = groups of 8 query heads
+        mp.a.H_q = c->h_pairs;  // pairs per sequence = groups of up to 8 query heads
         mp.n_q_heads = c->cfg.n_q_heads;
-        mp.groups_per_kv = c->cfg.n_q_heads / c->cfg.n_kv_heads / 8;
+        mp.heads_per_pair = mma_heads_per_pair(c->cfg);
+        mp.groups_per_kv = c->cfg.n_q_heads / c->cfg.n_kv_heads / mp.heads_per_pair;
         const int blk = lckv::kMmaWarps * 32;
         const size_t sm = lckv::kMmaSmemBytes;
         if (c->cfg.head_dim == 128)
@@ -728,7 +739,7 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     c->n_workers = sm * workers_per_sm(*cfg);
     c->kernel_kind = resolve_kernel_kind(*cfg);
     c->rows_per_tile = (c->kernel_kind == 2 ? lckv::kMmaSlotBytes : lckv::kAluSlotBytes) / (cfg->head_dim * 2);
-    c->h_pairs = c->kernel_kind == 2 ? cfg->n_q_heads / 8 : cfg->n_q_heads;
+    c->h_pairs = c->kernel_kind == 2 ? cfg->n_q_heads / mma_heads_per_pair(*cfg) : cfg->n_q_heads;
     make_layout(*cfg, c->plan.n_slots, c->n_workers, c->n_kv_layers, c->lay);
     if (dev_bytes < c->lay.total_bytes) { delete c; return LCKV_ENOMEM; }
     const float scale = cfg->softmax_scale > 0.f ? cfg->softmax_scale

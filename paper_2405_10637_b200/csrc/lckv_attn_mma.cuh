@@ -1,11 +1,13 @@
 // Decode attention, tensor-core kernel for grouped-query attention: the 8 query heads that share a
-// kv head form the N = 8 side of a dense bf16 m16n8k16 MMA tile.
+// kv head form the N = 8 side of a dense bf16 m16n8k16 MMA tile.  Groups of 2 ... 7 use the same
+// tile with zero queries in the unused columns (K and V are still read once per group, which is
+// what matters: the work is streaming them); larger groups are split into pairs of 8.
 //
 //   S^T [tokens x 8] = K [tokens x d] . Q^T [d x 8]        (tokens are the M dimension)
 //   O^T [d x 8]      = V^T [d x tokens] . P^T [tokens x 8]
 //
 // Work decomposition, per-warp copy ring, running-max softmax and the ticketed merge of split
-// pairs are those of the FP32-ALU kernel (lckv_attn_alu.cuh); a pair here is (sequence, group of 8
+// pairs are those of the FP32-ALU kernel (lckv_attn_alu.cuh); a pair here is (sequence, group of up to 8
 // query heads).  Differences: tiles arrive through 2-D tiled TMA with the 128-byte swizzle so that
 // ldmatrix reads them without bank conflicts; the probabilities are rounded to bf16 for the second
 // MMA (their sum is taken over the rounded values, so the weights stay normalised); a TMA box is
@@ -117,9 +119,11 @@ __device__ __forceinline__ void rcursor_next(RowCursor& c, const AttnParams& p, 
 }
 
 struct MmaParams {
-    AttnParams a;     // H_q here = pairs per sequence (groups of 8 query heads); see the launcher
+    AttnParams a;     // H_q here = pairs per sequence (groups of up to 8 query heads); see the launcher
     int32_t n_q_heads;  // real H_q, for addressing q / out / lse
-    int32_t groups_per_kv;  // groups of 8 query heads that share one kv head
+    int32_t groups_per_kv;  // pairs that share one kv head
+    int32_t heads_per_pair; // query heads of a pair: 8, or the whole group when it is smaller (the
+                            // other columns of the N = 8 tile then carry zero queries)
 };
 
 template <int D, bool PAGED = false>
@@ -143,6 +147,7 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
     const int H = p.H_q;  // pairs per sequence
     const uint32_t FULL = 0xffffffffu;
     const int g4 = lane >> 2, c4 = lane & 3;
+    const int HP = mp.heads_per_pair;
 
     const uint32_t smem0 = (smem_u32(smem_raw) + 1023u) & ~1023u;  // swizzle atoms are 1024 bytes
     const uint32_t ring = smem0 + warp * (NS * kMmaSlotBytes);
@@ -222,11 +227,12 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
     // Q^T fragments of the pair's 8 query heads: lane holds query g4, dims 2*c4 (+1) (+8) per k-step.
     uint32_t qb[KS][2];
     auto load_q = [&](const RowCursor& c) {
-        const uint16_t* qp = p.q + ((size_t)c.b * mp.n_q_heads + (size_t)c.h * 8 + g4) * D + 2 * c4;
+        const uint16_t* qp = p.q + ((size_t)c.b * mp.n_q_heads + (size_t)c.h * HP + g4) * D + 2 * c4;
+        const bool real = g4 < HP;
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
-            qb[ks][0] = __ldg(reinterpret_cast<const uint32_t*>(qp + ks * 16));
-            qb[ks][1] = __ldg(reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8));
+            qb[ks][0] = real ? __ldg(reinterpret_cast<const uint32_t*>(qp + ks * 16)) : 0u;
+            qb[ks][1] = real ? __ldg(reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8)) : 0u;
         }
     };
     load_q(cc);
@@ -428,16 +434,21 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
             }
             if (write_row) {
                 const float inv0 = 1.0f / l_tot[0], inv1 = 1.0f / l_tot[1];
-                const size_t row0 = (size_t)cc.b * mp.n_q_heads + (size_t)cc.h * 8;  // first q head
+                const size_t row0 = (size_t)cc.b * mp.n_q_heads + (size_t)cc.h * HP;  // first q head
+                const bool col0 = 2 * c4 < HP, col1 = 2 * c4 + 1 < HP;
                 if (p.out_f32) {
                     float* ob = static_cast<float*>(p.out);
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt) {
                         const int d0 = mt * 16 + g4;
-                        ob[(row0 + 2 * c4) * D + d0] = o[mt][0] * inv0;
-                        ob[(row0 + 2 * c4 + 1) * D + d0] = o[mt][1] * inv1;
-                        ob[(row0 + 2 * c4) * D + d0 + 8] = o[mt][2] * inv0;
-                        ob[(row0 + 2 * c4 + 1) * D + d0 + 8] = o[mt][3] * inv1;
+                        if (col0) {
+                            ob[(row0 + 2 * c4) * D + d0] = o[mt][0] * inv0;
+                            ob[(row0 + 2 * c4) * D + d0 + 8] = o[mt][2] * inv0;
+                        }
+                        if (col1) {
+                            ob[(row0 + 2 * c4 + 1) * D + d0] = o[mt][1] * inv1;
+                            ob[(row0 + 2 * c4 + 1) * D + d0 + 8] = o[mt][3] * inv1;
+                        }
                     }
                 } else {
                     // transpose the [dims x queries] fragments so a lane holds two adjacent dims of
@@ -447,13 +458,15 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
                     for (int mt = 0; mt < MT; ++mt) {
                         const uint32_t t0 = movmatrix_trans(cvt_bf16x2(o[mt][0] * inv0, o[mt][1] * inv1));
                         const uint32_t t1 = movmatrix_trans(cvt_bf16x2(o[mt][2] * inv0, o[mt][3] * inv1));
-                        *reinterpret_cast<uint32_t*>(ob + mt * 16) = t0;
-                        *reinterpret_cast<uint32_t*>(ob + mt * 16 + 8) = t1;
+                        if (g4 < HP) {
+                            *reinterpret_cast<uint32_t*>(ob + mt * 16) = t0;
+                            *reinterpret_cast<uint32_t*>(ob + mt * 16 + 8) = t1;
+                        }
                     }
                 }
                 if (p.lse && g4 == 0) {
-                    p.lse[row0 + 2 * c4] = (m_fin[0] + lg2(l_tot[0])) * 0.6931471805599453f;
-                    p.lse[row0 + 2 * c4 + 1] = (m_fin[1] + lg2(l_tot[1])) * 0.6931471805599453f;
+                    if (col0) p.lse[row0 + 2 * c4] = (m_fin[0] + lg2(l_tot[0])) * 0.6931471805599453f;
+                    if (col1) p.lse[row0 + 2 * c4 + 1] = (m_fin[1] + lg2(l_tot[1])) * 0.6931471805599453f;
                 }
             }
             m_run[0] = m_run[1] = -INFINITY;

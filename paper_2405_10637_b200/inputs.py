@@ -41,6 +41,9 @@ WORKLOADS = {
     "llama30b": Workload("llama30b", 4, 60, 52, 52, 128, 2, 1.0),
     # warmup-count / long-context sweep on the 7B shape
     "sweep7b": Workload("sweep7b", 5, 32, 32, 32, 128, 2, 1.0),
+    # a grouped-query layout outside the paper's models (groups of 4: 32 q heads, 8 kv heads, d_h 128),
+    # to time query groups smaller than the 8-wide tensor-core tile
+    "gqa4": Workload("gqa4", 6, 32, 32, 8, 128, 2, 1.0),
 }
 
 

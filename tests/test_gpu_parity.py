@@ -213,7 +213,7 @@ def test_repeatable_bitwise():
         assert np.array_equal(a, b)
 
 
-# ---- tensor-core kernel (query groups that are multiples of 8) -----------------------------------
+# ---- tensor-core kernel (grouped query heads) ------------------------------------------------------
 
 @pytest.mark.parametrize("d,Hq,Hkv", [(64, 32, 4), (128, 16, 2), (64, 32, 2), (128, 8, 1)])
 def test_mma_kernel_edge_lengths(d, Hq, Hkv):
@@ -222,6 +222,28 @@ def test_mma_kernel_edge_lengths(d, Hq, Hkv):
     assert c.cache.info.kernel_kind == 2
     for _ in range(3):
         c.step()
+    c.close()
+
+
+@pytest.mark.parametrize("d,Hq,Hkv", [(64, 8, 4), (128, 12, 4), (64, 16, 4), (128, 6, 1), (64, 14, 2)])
+@pytest.mark.parametrize("out_dtype", [0, 1])
+def test_mma_kernel_groups_smaller_than_8(d, Hq, Hkv, out_dtype):
+    """Query groups of 2, 3, 4, 6 and 7 use the tensor-core kernel with the unused columns of the
+    N = 8 tile zero: K and V are read once per group; only the real heads are written."""
+    lens = [0, 1, 15, 16, 17, 33, 64, 100, 257, 300]
+    c = Case(L=4, w=2, Hq=Hq, Hkv=Hkv, d=d, lens=lens, T_cap=303, seed=700 + d + Hq, std=0.5,
+             out_dtype=out_dtype)
+    assert c.cache.info.kernel_kind == 2
+    for _ in range(2):
+        c.step()
+    # lse of the real heads through the single-call entry
+    q = syn.randn_bf16((c.B, Hq, d), 5, std=0.5)
+    lse = torch.full((c.B, Hq), float("nan"), dtype=torch.float32, device=c.cache.device)
+    out = c.cache.lckv_decode_attention(0, lk.MODE_CONDENSED, q.to(c.cache.device), lse=lse)
+    torch.cuda.synchronize()
+    want, want_lse = orc.decode_attention(syn.bits(q), c.hK[0], c.hV[0], c.lens, 0, c.scale)
+    compare(out, want, "small group, single call")
+    assert np.abs(lse.cpu().numpy() - want_lse).max() < 2e-3
     c.close()
 
 
