@@ -221,7 +221,7 @@ void make_layout(const lckv_config_t& c, int n_slots, int n_workers, int n_kv_la
     y.pre_stride = (int)align_up((size_t)c.max_batch + 1, 64);
     y.off_pre = off;       off = align_up(off + 2 * (size_t)y.pre_stride * 4, A);
     y.off_start = off;     off = align_up(off + 2 * (size_t)n_workers * 4, A);
-    y.off_counters = off;  off = align_up(off + 2 * (size_t)n_workers * 4, A);  // two halves
+    y.off_counters = off;  off = align_up(off + 2 * 3 * (size_t)n_workers * 4, A);  // two halves of [pair tickets | chunk tickets]
     y.off_status = off;    off = align_up(off + 4, A);
     y.off_partials = off;
     off = align_up(off + 2 * 2 * (size_t)n_workers * partial_record_floats(c) * 4, A);  // two halves
@@ -387,7 +387,8 @@ int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out
     p.start_b = c->d_start + (size_t)mode * c->n_workers;
     // consecutive launches may overlap at their edges: alternate the split-K workspace halves
     p.partials = c->d_partials + (size_t)c->ws_parity * c->partials_half_floats;
-    p.counters = c->d_counters + (size_t)c->ws_parity * c->n_workers;
+    p.counters = c->d_counters + (size_t)c->ws_parity * 3 * c->n_workers;
+    p.counters2 = p.counters + c->n_workers;
     c->ws_parity ^= 1;
     p.status = c->d_status;
     p.T_cap = c->cfg.max_seq;
@@ -903,7 +904,7 @@ int lckv_cache_reset(lckv_cache_t* c, const int32_t* host_lens, int32_t batch, v
         for (int b = 0; b < batch; ++b) c->h_lens[b] = 0;
         if (!cuda_ok(cudaMemsetAsync(c->d_lens, 0, (size_t)batch * 4, st))) return LCKV_ECUDA;
     }
-    if (!cuda_ok(cudaMemsetAsync(c->d_counters, 0, 2 * (size_t)c->n_workers * 4, st))) return LCKV_ECUDA;
+    if (!cuda_ok(cudaMemsetAsync(c->d_counters, 0, 2 * 3 * (size_t)c->n_workers * 4, st))) return LCKV_ECUDA;
     if (!cuda_ok(cudaMemsetAsync(c->d_status, 0, 4, st))) return LCKV_ECUDA;
     return sync_page_table(c, st);
 }
@@ -1342,6 +1343,7 @@ extern "C" int lckv_decode_attention_static(const void* k, const void* v, const 
     p.start_b = d_start + (size_t)mode * n_workers;
     p.partials = reinterpret_cast<float*>(base + kStOffPartials);
     p.counters = d_counters;
+    p.counters2 = nullptr;
     p.status = d_status;
     p.T_cap = max_seq;
     p.B = batch;

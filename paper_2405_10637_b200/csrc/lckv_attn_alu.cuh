@@ -48,6 +48,7 @@ struct AttnParams {
     const int32_t* start_b;   // [n_workers] for this mode
     float* partials;          // [2 * n_workers][D + 4]
     int32_t* counters;        // [n_workers], zero between launches
+    int32_t* counters2;      // [2 * n_workers] tickets of first-level merge chunks (tensor-core kernel; may be null)
     int32_t* status;          // device status word
     int64_t T_cap;
     int32_t B, H_q, H_kv, mode, n_workers, out_f32;

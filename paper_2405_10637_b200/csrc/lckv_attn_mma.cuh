@@ -32,6 +32,8 @@ constexpr int kMmaSlots = LCKV_MMA_SLOTS;
 #endif
 constexpr int kMmaSlotBytes = LCKV_MMA_SLOT_BYTES;
 constexpr int kMmaSmemBytes = kMmaWarps * kMmaSlots * (kMmaSlotBytes + 8) + 1024;  // + alignment slack
+constexpr int kMmaTreeMin = 24;   // pairs split over more workers than this are merged in two levels
+constexpr int kMmaChunk = 16;     // contributors per first-level chunk
 
 __device__ __forceinline__ void ldmatrix_x4(uint32_t addr, uint32_t& r0, uint32_t& r1, uint32_t& r2,
                                             uint32_t& r3)
@@ -381,19 +383,17 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
                 }
                 __threadfence();
                 __syncwarp();
-                int ticket = 0;
-                if (lane == 0) ticket = atomicAdd(p.counters + c_first, 1);
-                ticket = __shfl_sync(FULL, ticket, 0);
-                if (ticket == (int)(c_last - c_first)) {
-                    __threadfence();
-                    const uint64_t lo_first = (uint64_t)c_first * total / n_eff;
-                    const float* rec0 = p.partials + (size_t)(2 * c_first) * REC;
-                    const int first_odd = (gs != lo_first) ? 1 : 0;
-                    const int n_parts = (int)(c_last - c_first) + 1;
+                // Merge of n records in a fixed order: record i is the one of worker
+                // first_w + i * step (its second record if i == 0 and first_slot is set).  Record
+                // addresses do not depend on loaded data, so the unrolled loops keep several L2 round
+                // trips in flight.  Leaves the merged (unnormalised) values in o, l_tot, m_fin.
+                auto merge_records = [&](int n, uint32_t first_w, int step, int first_slot) {
+                    const float* rec0 = p.partials + (size_t)(2 * first_w) * REC;
+                    const size_t rstride = (size_t)(2 * step) * REC;
                     float M[2] = {-INFINITY, -INFINITY};
 #pragma unroll 4
-                    for (int i = 0; i < n_parts; ++i) {
-                        const float* r = rec0 + (size_t)(2 * i + (i == 0 ? first_odd : 0)) * REC;
+                    for (int i = 0; i < n; ++i) {
+                        const float* r = rec0 + (size_t)i * rstride + (i == 0 ? (size_t)first_slot * REC : 0);
                         const float2 mm = __ldcg(reinterpret_cast<const float2*>(r + D * 8) + c4);
                         M[0] = fmaxf(M[0], mm.x);
                         M[1] = fmaxf(M[1], mm.y);
@@ -405,8 +405,8 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
 #pragma unroll
                         for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
 #pragma unroll 2
-                    for (int i = 0; i < n_parts; ++i) {
-                        const float* r = rec0 + (size_t)(2 * i + (i == 0 ? first_odd : 0)) * REC;
+                    for (int i = 0; i < n; ++i) {
+                        const float* r = rec0 + (size_t)i * rstride + (i == 0 ? (size_t)first_slot * REC : 0);
                         const float2 mm = __ldcg(reinterpret_cast<const float2*>(r + D * 8) + c4);
                         const float2 ll = __ldcg(reinterpret_cast<const float2*>(r + D * 8 + 8) + c4);
                         const float w0 = ex2(mm.x - M[0]);
@@ -428,8 +428,48 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
                         for (int i = 0; i < 4; ++i) o[mt][i] = acc[mt][i];
                     l_tot[0] = Ls[0]; l_tot[1] = Ls[1];
                     m_fin[0] = M[0]; m_fin[1] = M[1];
-                    write_row = true;
-                    if (lane == 0) p.counters[c_first] = 0;
+                };
+                const uint64_t lo_first = (uint64_t)c_first * total / n_eff;
+                const int first_odd = (gs != lo_first) ? 1 : 0;   // which record of c_first belongs to this pair
+                const int n_parts = (int)(c_last - c_first) + 1;
+                // Few parts: the contributor that arrives last merges them all.  Many parts (few
+                // pairs, long sequences): two levels - the contributors of a pair form chunks of
+                // kMmaChunk consecutive workers; the last arriver of a chunk merges the chunk's records
+                // into the record of the chunk's first worker, and the last chunk to finish merges
+                // the chunk records.  Same fixed order either way.
+                const bool two_level = n_parts > kMmaTreeMin && p.counters2 != nullptr;
+                const int k = (int)((uint32_t)w - c_first);          // this contributor's index in the pair
+                const int ck = (k / kMmaChunk) * kMmaChunk;          // its chunk's first index
+                const uint32_t cw = c_first + (uint32_t)ck;          // chunk's first worker
+                const int cslot = (ck == 0) ? first_odd : 0;
+                const int n_chunks = (n_parts + kMmaChunk - 1) / kMmaChunk;
+                // first round: chunk level (two-level) or pair level (direct); second round: pair level
+                int32_t* tk = two_level ? p.counters2 + 2 * cw + cslot : p.counters + c_first;
+                int n = two_level ? min(kMmaChunk, n_parts - ck) : n_parts;
+                uint32_t fw = two_level ? cw : c_first;
+                int step = 1, fslot = two_level ? cslot : first_odd;
+                for (int round = two_level ? 0 : 1; round < 2; ++round) {
+                    int ticket = 0;
+                    if (lane == 0) ticket = atomicAdd(tk, 1);
+                    ticket = __shfl_sync(FULL, ticket, 0);
+                    if (ticket != n - 1) break;          // someone else arrives later and merges
+                    __threadfence();
+                    merge_records(n, fw, step, fslot);
+                    if (lane == 0) *tk = 0;              // ready for the next launch
+                    if (round == 1) { write_row = true; break; }
+                    // the chunk's result becomes the record of the chunk's first worker
+                    float* crec = p.partials + (size_t)(2 * cw + cslot) * REC;
+#pragma unroll
+                    for (int mt = 0; mt < MT; ++mt)
+                        reinterpret_cast<float4*>(crec)[mt * 32 + lane] =
+                            make_float4(o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
+                    if (g4 == 0) {
+                        crec[D * 8 + 2 * c4] = m_fin[0];     crec[D * 8 + 2 * c4 + 1] = m_fin[1];
+                        crec[D * 8 + 8 + 2 * c4] = l_tot[0]; crec[D * 8 + 8 + 2 * c4 + 1] = l_tot[1];
+                    }
+                    __threadfence();
+                    __syncwarp();
+                    tk = p.counters + c_first; n = n_chunks; fw = c_first; step = kMmaChunk; fslot = first_odd;
                 }
             }
             if (write_row) {

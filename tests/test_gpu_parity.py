@@ -263,6 +263,23 @@ def test_mma_kernel_single_long_pair():
     c.close()
 
 
+@pytest.mark.parametrize("d,Hq,Hkv", [(128, 16, 2), (64, 8, 2), (128, 8, 1)])
+def test_mma_kernel_few_pairs_split_over_many_workers(d, Hq, Hkv):
+    """Few (sequence, kv head) pairs and long sequences: a pair is split over tens to hundreds of
+    workers and its parts are merged in two levels (chunks of contributors, then chunk results)."""
+    lens = [30000, 4100, 123]
+    c = Case(L=2, w=0, Hq=Hq, Hkv=Hkv, d=d, lens=lens, T_cap=30010, seed=77 + d, std=0.25, poison=False)
+    assert c.cache.info.kernel_kind == 2
+    c.step(); c.step()
+    # twice the same call: the merge order is fixed, so the results repeat bit for bit
+    q = syn.randn_bf16((3, Hq, d), 9, std=0.25).to(c.cache.device)
+    a = c.cache.lckv_decode_attention(0, lk.MODE_CONDENSED, q).clone()
+    b = c.cache.lckv_decode_attention(0, lk.MODE_CONDENSED, q)
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
+    c.close()
+
+
 def test_tinyllama_shape_stack():
     """22 layers, 32 q heads, 4 kv heads, d_h 64, w = 2, values scaled by 1/sqrt(d_h) (rel-L2 binds)."""
     lens = [512, 513, 1024, 1535, 700, 511, 33, 1200]
