@@ -36,6 +36,8 @@ constexpr int kAluWarps = LCKV_ALU_WARPS;  // workers per CTA
 constexpr int kAluSlots = LCKV_ALU_SLOTS;  // ring slots per worker
 constexpr int kAluSlotBytes = LCKV_ALU_SLOT_BYTES;  // one tile of K or of V (a multiple of 4 KB)
 constexpr int kAluSmemBytes = kAluWarps * kAluSlots * (kAluSlotBytes + 8);
+constexpr int kAluTreeMin = 24;   // pairs split over more workers than this are merged in two levels
+constexpr int kAluChunk = 16;     // contributors per first-level chunk
 
 struct AttnParams {
     const uint16_t* K;        // [B_max, H_kv, T_cap, D] bf16
@@ -407,30 +409,25 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
                 if (lane == 0) { rec[D] = m_fin; rec[D + 1] = l_tot; }
                 __threadfence();
                 __syncwarp();
-                int ticket = 0;
-                if (lane == 0) ticket = atomicAdd(p.counters + c_first, 1);
-                ticket = __shfl_sync(FULL, ticket, 0);
-                if (ticket == (int)(c_last - c_first)) {
-                    // Last contributor: merge every part in worker order (fixed summation order).
-                    // Record addresses do not depend on loaded data, so the unrolled loops keep
-                    // several L2 round trips in flight.
-                    __threadfence();
-                    const uint64_t lo_first = (uint64_t)c_first * total / n_eff;
-                    const float* rec0 = p.partials + (size_t)(2 * c_first) * REC;
-                    const int first_odd = (gs != lo_first) ? 1 : 0;  // which record of c_first
-                    const int n_parts = (int)(c_last - c_first) + 1;
+                // Merge of n records in a fixed order: record i is the one of worker
+                // first_w + i * step (its second record if i == 0 and first_slot is set).  Record
+                // addresses do not depend on loaded data, so the unrolled loops keep several L2 round
+                // trips in flight.  Leaves the merged (unnormalised) values in o, l_tot, m_fin.
+                auto merge_records = [&](int n, uint32_t first_w, int step, int first_slot) {
+                    const float* rec0 = p.partials + (size_t)(2 * first_w) * REC;
+                    const size_t rstride = (size_t)(2 * step) * REC;
                     float M = -INFINITY;
 #pragma unroll 4
-                    for (int i = 0; i < n_parts; ++i) {
-                        const float* r = rec0 + (size_t)(2 * i + (i == 0 ? first_odd : 0)) * REC;
+                    for (int i = 0; i < n; ++i) {
+                        const float* r = rec0 + (size_t)i * rstride + (i == 0 ? (size_t)first_slot * REC : 0);
                         M = fmaxf(M, __ldcg(r + D));
                     }
                     float Lsum = 0.f, acc[8];
 #pragma unroll
                     for (int k = 0; k < 8; ++k) acc[k] = 0.f;
 #pragma unroll 4
-                    for (int i = 0; i < n_parts; ++i) {
-                        const float* r = rec0 + (size_t)(2 * i + (i == 0 ? first_odd : 0)) * REC;
+                    for (int i = 0; i < n; ++i) {
+                        const float* r = rec0 + (size_t)i * rstride + (i == 0 ? (size_t)first_slot * REC : 0);
                         const float2 ml = __ldcg(reinterpret_cast<const float2*>(r + D));
                         const float wgt = ex2(ml.x - M);
                         Lsum = fmaf(ml.y, wgt, Lsum);
@@ -448,8 +445,44 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
                     for (int k = 0; k < 8; ++k) o[k] = acc[k];
                     l_tot = Lsum;
                     m_fin = M;
-                    write_row = true;
-                    if (lane == 0) p.counters[c_first] = 0;  // ready for the next launch
+                };
+                const uint64_t lo_first = (uint64_t)c_first * total / n_eff;
+                const int first_odd = (gs != lo_first) ? 1 : 0;  // which record of c_first belongs to this pair
+                const int n_parts = (int)(c_last - c_first) + 1;
+                // Few parts: the contributor that arrives last merges them all.  Many parts (few
+                // pairs, long sequences): two levels - the contributors of a pair form chunks of
+                // kAluChunk consecutive workers; the last arriver of a chunk merges the chunk's records
+                // into the record of the chunk's first worker, and the last chunk to finish merges
+                // the chunk records.  Same fixed order either way.
+                const bool two_level = n_parts > kAluTreeMin && p.counters2 != nullptr;
+                const int kk = (int)((uint32_t)w - c_first);         // this contributor's index in the pair
+                const int ck = (kk / kAluChunk) * kAluChunk;         // its chunk's first index
+                const uint32_t cw = c_first + (uint32_t)ck;          // chunk's first worker
+                const int cslot = (ck == 0) ? first_odd : 0;
+                int32_t* tk = two_level ? p.counters2 + 2 * cw + cslot : p.counters + c_first;
+                int n = two_level ? min(kAluChunk, n_parts - ck) : n_parts;
+                uint32_t fw = two_level ? cw : c_first;
+                int step = 1, fslot = two_level ? cslot : first_odd;
+                for (int round = two_level ? 0 : 1; round < 2; ++round) {
+                    int ticket = 0;
+                    if (lane == 0) ticket = atomicAdd(tk, 1);
+                    ticket = __shfl_sync(FULL, ticket, 0);
+                    if (ticket != n - 1) break;          // someone else arrives later and merges
+                    __threadfence();
+                    merge_records(n, fw, step, fslot);
+                    if (lane == 0) *tk = 0;              // ready for the next launch
+                    if (round == 1) { write_row = true; break; }
+                    // the chunk's result becomes the record of the chunk's first worker
+                    float* crec = p.partials + (size_t)(2 * cw + cslot) * REC;
+                    if (lane < LPR) {
+                        reinterpret_cast<float4*>(crec)[2 * lane] = make_float4(o[0], o[1], o[2], o[3]);
+                        reinterpret_cast<float4*>(crec)[2 * lane + 1] = make_float4(o[4], o[5], o[6], o[7]);
+                    }
+                    if (lane == 0) { crec[D] = m_fin; crec[D + 1] = l_tot; }
+                    __threadfence();
+                    __syncwarp();
+                    tk = p.counters + c_first; n = (n_parts + kAluChunk - 1) / kAluChunk; fw = c_first;
+                    step = kAluChunk; fslot = first_odd;
                 }
             }
             if (write_row) {

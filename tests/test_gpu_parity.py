@@ -94,6 +94,22 @@ def test_single_long_sequence_split_over_many_workers():
     c.close()
 
 
+@pytest.mark.parametrize("d,H", [(128, 2), (64, 3)])
+def test_few_pairs_split_over_many_workers_two_level_merge(d, H):
+    """Multi-head attention with very few (sequence, head) pairs and long sequences: a pair is split
+    over hundreds of workers and its parts are merged in two levels; results repeat bit for bit."""
+    lens = [30000, 4100]
+    c = Case(L=2, w=0, Hq=H, Hkv=H, d=d, lens=lens, T_cap=30010, seed=177 + d, std=0.25, poison=False)
+    assert c.cache.info.kernel_kind == 1
+    c.step(); c.step()
+    q = syn.randn_bf16((2, H, d), 9, std=0.25).to(c.cache.device)
+    a = c.cache.lckv_decode_attention(0, lk.MODE_CONDENSED, q).clone()
+    b = c.cache.lckv_decode_attention(0, lk.MODE_CONDENSED, q)
+    torch.cuda.synchronize()
+    assert torch.equal(a, b)
+    c.close()
+
+
 def test_decode_attention_entry_lse_and_single_key_exactness():
     """Per-layer entry point: log-sum-exp output; one visible key gives o = v_0 bit-exactly."""
     B, H, d, T = 3, 4, 128, 50
