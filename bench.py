@@ -40,7 +40,7 @@ NOMINAL_HBM_GBS = 8000.0
 NCU_CAPTURES = {
     "attn_alu_kernel": {
         "source": "profiles/attn_alu_kernel_llama7b_b8_ncu_full.md",
-        "alg_in": 283.9e6 - 65536, "read": 284.01e6, "write": 4.42e6, "out": 65536,
+        "alg_in": 283.9e6 - 65536, "read": 284.00e6, "write": 3.46e6, "out": 65536,
         "applies": lambda a: a.workload in ("llama7b", "llama30b", "sweep7b") and not a.page_rows,
     },
     "attn_mma_kernel": {
