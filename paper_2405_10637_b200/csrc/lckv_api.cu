@@ -1002,8 +1002,9 @@ int lckv_project_append_kv(lckv_cache_t* c, int32_t slot, const void* x, int32_t
     if (int rc = ensure_pages(c, batch, 1)) return rc;
     if (int rc = sync_page_table(c, st)) return rc;
 
-    int NB = 16;
-    while (NB < batch && NB < 256) NB *= 2;
+    // batch tile = N of the MMA: any multiple of 16 up to 256; equal tiles when the batch needs several
+    const int n_btiles = (batch + 255) / 256;
+    const int NB = ((batch + n_btiles - 1) / n_btiles + 15) / 16 * 16;
     int n_stages = (192 * 1024) / lckv::proj_stage_bytes(NB);
     if (n_stages > 8) n_stages = 8;
     CUtensorMap tx, tk, tv;

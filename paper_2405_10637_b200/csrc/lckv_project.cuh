@@ -48,7 +48,7 @@ struct ProjParams {
     int64_t T_cap;
     int32_t pt_stride, page_shift;
     int32_t B, H_kv, D, d_model;
-    int32_t NB;               // batch tile = N of the MMA (16, 32, 64, 128, 256)
+    int32_t NB;               // batch tile = N of the MMA (a multiple of 16, at most 256)
     int32_t n_stages;
     int32_t n_sink;
     int32_t k_tiles;          // feature tiles of K; tiles k_tiles .. 2*k_tiles-1 belong to V
@@ -112,7 +112,8 @@ project_kv_kernel(const ProjParams p, const __grid_constant__ CUtensorMap tmX,
     const uint32_t rank = KS > 1 ? cluster_ctarank() : 0u;
     const int n_k = p.d_model / kProjBK / KS;       // this CTA's k-steps
     const int k_first = (int)rank * n_k;
-    const uint32_t tm_cols = NB < 32 ? 32u : (uint32_t)NB;
+    uint32_t tm_cols = 32;                      // allocation: a power of two >= NB
+    while ((int)tm_cols < NB) tm_cols *= 2;
 
     if (tid == 0) {
         for (int s = 0; s < NS; ++s) { mbar_init(bFull + 8 * s, 1); mbar_init(bEmpty + 8 * s, 1); }
