@@ -171,6 +171,17 @@ int lckv_cache_lengths(const lckv_cache_t* cache, int32_t* host_out, int32_t bat
  */
 int lckv_cache_status(const lckv_cache_t* cache, int32_t* host_status, void* stream);
 
+/*
+ * Sets how many polls a device-side wait on a copy may take in the decode attention kernels
+ * before the kernel gives up (default 2^18; one poll parks the warp for up to 20 us).  A wait that
+ * runs out sets the status word to LCKV_ETIMEOUT, lets the copies still in flight land (a second,
+ * fixed bound) and returns; that launch's outputs and the merge tickets are then undefined until
+ * lckv_cache_reset.  0 makes the first wait of every worker give up at once: a way to exercise the
+ * timeout path without anything actually hanging.  Takes effect from the next launch (a captured
+ * step is dropped and captured again).  EINVAL on null.
+ */
+int lckv_cache_set_wait_limit(lckv_cache_t* cache, uint32_t polls);
+
 /* Device pointers of slot `slot`'s K and V tensors [B_max, H_kv, T_cap, d_h] bf16 (for filling
  * a cache with a prompt's keys and values, or inspecting it).  EINVAL on bad slot / null. */
 int lckv_cache_slot_ptrs(const lckv_cache_t* cache, int32_t slot, void** k, void** v);
@@ -351,16 +362,21 @@ int lckv_prefill_iteration(lckv_cache_t* cache, const void* const* q_layers,
  *
  * Set-up: the first call on each device looks up the array's device address
  * and raises the kernel's shared-memory limit; make that first call outside
- * any stream capture.  Later calls on that device only enqueue work.
+ * any stream capture (it is refused with EINVAL inside one); the set-up is
+ * guarded, so first calls from several host threads are safe.  Later calls on that device only enqueue work.
  * Sharing: all calls on a device use the same scratch.  Calls are safe one
  * after another on one stream (the merge tickets are cleared at the start of
  * each call); calls that may overlap on the GPU - different streams, or a
  * cache-based call is unaffected but two static calls are - race on it and
- * give undefined results.  The lengths are read on the device, so a length
- * beyond max_seq cannot be refused here: the caller guarantees
- * 0 <= lens[b] and lens[b] + mode <= max_seq.
+ * give undefined results.  The lengths are read on the device, so a bad length
+ * cannot be refused here: the visible count is clamped to [0, max_seq] (nothing
+ * outside the tensors is read), but the result for such a sequence is not what
+ * the caller meant; keep 0 <= lens[b] and lens[b] + mode <= max_seq.
  * This call performs no cudaMalloc/cudaFree and uses no allocating library.
- * Errors: EINVAL (null pointer, bad shape or mode), ESTATICLIMIT, ECUDA.
+ * Errors: EINVAL (null pointer; k, v, q or out not 16-byte aligned; lens, lse
+ * or dev_status not 4-byte aligned; bad shape or mode; a first call on a device
+ * made while `stream` is capturing), ESTATICLIMIT, ECUDA.  Argument errors are
+ * found before any CUDA call is made.
  */
 #define LCKV_STATIC_MAX_BATCH 4096
 #define LCKV_STATIC_MAX_SMS 256
@@ -370,6 +386,21 @@ int lckv_decode_attention_static(const void* k, const void* v, const int32_t* le
                                  int32_t batch, int32_t n_q_heads, int32_t n_kv_heads,
                                  int32_t head_dim, int64_t max_seq, int32_t mode,
                                  float softmax_scale, int32_t out_dtype, void* stream);
+
+/*
+ * Measurement helper (the paper has no counterpart): a read-only stream over `bytes` of device
+ * memory at `src` (16-byte aligned), to learn the read bandwidth this GPU reaches when the bytes are
+ * only read - the ceiling of the read-dominated attention kernels, which a read + write copy does
+ * not show.  kind 0: independent 16-byte loads from every thread; kind 2: 32-byte loads
+ * (src 32-byte aligned) marked evict-first; kind 1: 8 KB bulk copies into
+ * per-warp shared-memory rings, the way the attention kernels stream K and V (bytes beyond the last
+ * whole 8 KB are not read).  *dev_sum (device uint32, not cleared) receives a checksum so that the
+ * reads cannot be optimised away: kinds 0 and 2 add the wrapped sum of all 32-bit words, kind 1 the first
+ * word of every piece.  *dev_status (device int32) is set to LCKV_ETIMEOUT if a bounded wait of kind 1
+ * runs out.  Time it with events on `stream`.  Errors: EINVAL, ECUDA.
+ */
+int lckv_read_stream_probe(const void* src, size_t bytes, int32_t kind, uint32_t* dev_sum,
+                           int32_t* dev_status, void* stream);
 
 /* Short English name of a status code. */
 const char* lckv_status_string(int status);

@@ -43,6 +43,7 @@ SIGNATURES = {
     "lckv_cache_reset": (C.c_int, [_vp, _i32p, _i32, _vp]),
     "lckv_cache_lengths": (C.c_int, [_vp, _i32p, _i32, _vp]),
     "lckv_cache_status": (C.c_int, [_vp, _i32p, _vp]),
+    "lckv_cache_set_wait_limit": (C.c_int, [_vp, C.c_uint32]),
     "lckv_cache_slot_ptrs": (C.c_int, [_vp, _i32, _vpp, _vpp]),
     "lckv_cache_page_table": (C.c_int, [_vp, _i32p, _i32p]),
     "lckv_append_kv": (C.c_int, [_vp, _i32, _vp, _vp, _i32, _i32, _vp]),
@@ -55,6 +56,7 @@ SIGNATURES = {
     "lckv_prefill_iteration": (C.c_int, [_vp, _vpp, _vpp, _vpp, _vpp, _i32, _i32, _vp]),
     "lckv_decode_attention_static": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32,
                                               _i32, C.c_int64, _i32, C.c_float, _i32, _vp]),
+    "lckv_read_stream_probe": (C.c_int, [_vp, C.c_size_t, _i32, _vp, _vp, _vp]),
     "lckv_status_string": (C.c_char_p, [C.c_int]),
     "lckv_last_cuda_error": (C.c_int, []),
 }
@@ -145,6 +147,13 @@ def lckv_decode_attention_static(k, v, lens, q, out, mode, lse=None, dev_status=
     return out
 
 
+def lckv_read_stream_probe(src, nbytes, kind, dev_sum, dev_status, stream=None):
+    """Read-only stream over the first nbytes of the CUDA tensor `src`; dev_sum (uint32/int32 [1]) and
+    dev_status (int32 [1]) are CUDA tensors."""
+    _chk(lib().lckv_read_stream_probe(_ptr(src), nbytes, kind, _ptr(dev_sum), _ptr(dev_status),
+                                      _stream(stream)), "lckv_read_stream_probe")
+
+
 class Cache:
     """Owner of one lckv_cache_t and of the torch buffer behind it."""
 
@@ -197,6 +206,9 @@ class Cache:
         s = C.c_int32(0)
         _chk(lib().lckv_cache_status(self.h, C.byref(s), _stream(stream)), "lckv_cache_status")
         return s.value
+
+    def lckv_cache_set_wait_limit(self, polls):
+        _chk(lib().lckv_cache_set_wait_limit(self.h, polls), "lckv_cache_set_wait_limit")
 
     def lckv_cache_slot_ptrs(self, slot):
         k, v = C.c_void_p(), C.c_void_p()

@@ -1,10 +1,12 @@
 // Host runtime and C ABI of the LCKV decode-attention library (see include/lckv.h).
 #include <cuda_runtime.h>
 
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
+#include <mutex>
 #include <new>
 #include <vector>
 
@@ -14,6 +16,7 @@
 #include "lckv_project.cuh"
 #include "lckv_prefill.cuh"
 #include "lckv_prefill_tc5.cuh"
+#include "lckv_probe.cuh"
 #include "lckv_small_kernels.cuh"
 
 namespace {
@@ -103,6 +106,7 @@ struct lckv_cache {
     bool pt_dirty;
     int prefill_tc5;                      // 1: prompt encoding on tcgen05, 0: mma.sync kernel
     double l2_keep_bytes;                 // how much of a re-read slot to hold in L2 (0 = off)
+    uint32_t wait_limit;                  // polls a device-side wait on a copy may take
     int ws_parity;                        // which half of the split-K workspace the next launch uses
     size_t partials_half_floats;          // floats in one half of the partial records
     // CUDA graph of one step, valid for the argument pointers it was captured with
@@ -400,6 +404,7 @@ int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out
     p.out_f32 = c->cfg.out_dtype;
     p.scale_log2 = c->scale_log2;
     p.early_kv = early ? 1 : 0;
+    p.wait_limit = c->wait_limit;
     p.l2_keep = l2_keep;
     p.page_table = c->d_pt;
     p.pt_stride = c->pt_stride;
@@ -781,6 +786,7 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
         c->prefill_tc5 = !(env && env[0] == 'm');
     }
     c->ws_parity = 0;
+    c->wait_limit = lckv::kDefaultWaitLimit;
     c->partials_half_floats = 2 * (size_t)c->n_workers * partial_record_floats(*cfg);
     c->graph_exec = nullptr;
 
@@ -925,6 +931,14 @@ int lckv_cache_status(const lckv_cache_t* c, int32_t* host_status, void* stream)
     if (!cuda_ok(cudaMemcpyAsync(host_status, c->d_status, 4, cudaMemcpyDeviceToHost, st)))
         return LCKV_ECUDA;
     return cuda_ok(cudaStreamSynchronize(st)) ? LCKV_OK : LCKV_ECUDA;
+}
+
+int lckv_cache_set_wait_limit(lckv_cache_t* c, uint32_t polls)
+{
+    if (!c) return LCKV_EINVAL;
+    c->wait_limit = polls;
+    drop_graph(c);   // a captured step carries the old limit in its kernel arguments
+    return LCKV_OK;
 }
 
 int lckv_cache_slot_ptrs(const lckv_cache_t* c, int32_t slot, void** k, void** v)
@@ -1138,6 +1152,9 @@ int lckv_layer_stack_step_host(lckv_cache_t* c, const void* const* q_host, void*
         c->ev.push_back(e);
     }
     cudaEvent_t ev_start = c->ev[0], ev_kv = c->ev[1], ev_out = c->ev[2];
+    // everything that can refuse the step comes before the first copy is queued
+    if (int rc = ensure_pages(c, batch, 1)) return rc;
+    if (int rc = sync_page_table(c, st)) return rc;
     // staging buffers are free once everything queued on the caller's stream so far has run
     if (!cuda_ok(cudaEventRecord(ev_start, st)) || !cuda_ok(cudaStreamWaitEvent(c->s_in, ev_start, 0)))
         return LCKV_ECUDA;
@@ -1162,8 +1179,6 @@ int lckv_layer_stack_step_host(lckv_cache_t* c, const void* const* q_host, void*
         hooks.wait_before[l0] = c->ev[3 + 2 * k];
         hooks.record_after[l0 + n - 1] = c->ev[4 + 2 * k];
     }
-    if (int rc = ensure_pages(c, batch, 1)) return rc;
-    if (int rc = sync_page_table(c, st)) return rc;
     if (int rc = enqueue_step(c, dq.data(), dout.data(), dk.data(), dv.data(), batch, st, &hooks)) return rc;
     mirror_advance(c, batch);
     for (int k = 0; k < n_chunks; ++k) {
@@ -1228,6 +1243,39 @@ int lckv_prefill_iteration(lckv_cache_t* c, const void* const* q_layers, void* c
     return LCKV_OK;
 }
 
+int lckv_read_stream_probe(const void* src, size_t bytes, int32_t kind, uint32_t* dev_sum,
+                           int32_t* dev_status, void* stream)
+{
+    if (!src || !dev_sum || !dev_status || bytes < 16) return LCKV_EINVAL;
+    if (((uintptr_t)src & 15) || ((uintptr_t)dev_sum & 3) || ((uintptr_t)dev_status & 3)) return LCKV_EINVAL;
+    if (kind < 0 || kind > 2 || (kind == 2 && ((uintptr_t)src & 31))) return LCKV_EINVAL;
+    int sm = 0;
+    if (int rc = device_sm_count(&sm)) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    if (kind == 0) {
+        // 8 resident blocks of 256 threads per SM: 16 KB of loads in flight per SM and loop trip
+        lckv::read_stream_ldg_kernel<<<sm * 8, lckv::kProbeThreads, 0, st>>>(
+            static_cast<const uint4*>(src), (uint64_t)(bytes / 16), dev_sum);
+    } else if (kind == 2) {
+        lckv::read_stream_ldg32_kernel<<<sm * 8, lckv::kProbeThreads, 0, st>>>(
+            static_cast<const uint8_t*>(src), (uint64_t)(bytes / 32), dev_sum);
+    } else {
+        static std::once_flag once[64];
+        int dev = 0;
+        if (!cuda_ok(cudaGetDevice(&dev)) || dev < 0 || dev >= 64) return LCKV_ECUDA;
+        bool ok = true;
+        std::call_once(once[dev], [&] {
+            ok = cuda_ok(cudaFuncSetAttribute(lckv::read_stream_bulk_kernel,
+                                              cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                              lckv::kProbeSmemBytes));
+        });
+        if (!ok) return LCKV_ECUDA;
+        lckv::read_stream_bulk_kernel<<<sm, lckv::kProbeThreads, lckv::kProbeSmemBytes, st>>>(
+            static_cast<const uint8_t*>(src), (uint64_t)(bytes / lckv::kProbePiece), dev_sum, dev_status);
+    }
+    return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
+}
+
 const char* lckv_status_string(int s)
 {
     switch (s) {
@@ -1268,10 +1316,13 @@ static_assert(kStOffStart % 256 == 0 && kStOffCounters % 256 == 0 && kStOffParti
 static __device__ __align__(256) unsigned char g_static_scratch[LCKV_STATIC_SCRATCH_BYTES];
 
 constexpr int kMaxDevices = 64;
-unsigned char* g_static_ptr[kMaxDevices];   // device address of the array, per device
+std::mutex g_static_mutex;                            // guards the per-device set-up below
+std::atomic<unsigned char*> g_static_ptr[kMaxDevices];  // device address of the array, per device;
+                                                      // published last, after g_static_sms
 int g_static_sms[kMaxDevices];
 
-// Once per device, with that device current: resolve the array's device address.
+// Once per device, with that device current: resolve the array's device address.  Called with
+// g_static_mutex held.
 int static_setup(int dev)
 {
     void* ptr = nullptr;
@@ -1287,7 +1338,7 @@ int static_setup(int dev)
                                       lckv::kAluSmemBytes)))
         return LCKV_ECUDA;
     g_static_sms[dev] = sms;
-    g_static_ptr[dev] = static_cast<unsigned char*>(ptr);
+    g_static_ptr[dev].store(static_cast<unsigned char*>(ptr), std::memory_order_release);
     return LCKV_OK;
 }
 
@@ -1301,6 +1352,10 @@ extern "C" int lckv_decode_attention_static(const void* k, const void* v, const 
                                             void* stream)
 {
     if (!k || !v || !lens || !q || !out) return LCKV_EINVAL;
+    // k, v move by 16-byte bulk copies, q and out by 128-bit loads and stores: a pointer off that
+    // grid would fault on the device, so it is refused here
+    if (((uintptr_t)k | (uintptr_t)v | (uintptr_t)q | (uintptr_t)out) & 15) return LCKV_EINVAL;
+    if (((uintptr_t)lens | (uintptr_t)lse | (uintptr_t)dev_status) & 3) return LCKV_EINVAL;
     if (batch < 1 || n_q_heads < 1 || n_kv_heads < 1 || n_q_heads % n_kv_heads) return LCKV_EINVAL;
     if (head_dim != 64 && head_dim != 128) return LCKV_EINVAL;
     if (max_seq < 1 || max_seq > 0x7fffffff) return LCKV_EINVAL;
@@ -1312,13 +1367,21 @@ extern "C" int lckv_decode_attention_static(const void* k, const void* v, const 
     int dev = 0;
     if (!cuda_ok(cudaGetDevice(&dev))) return LCKV_ECUDA;
     if (dev < 0 || dev >= kMaxDevices) return LCKV_ESTATICLIMIT;
-    if (!g_static_ptr[dev])
-        if (int rc = static_setup(dev)) return rc;
+    cudaStream_t st = static_cast<cudaStream_t>(stream);
+    unsigned char* base = g_static_ptr[dev].load(std::memory_order_acquire);
+    if (!base) {
+        // The set-up calls are not stream work and must not land in a capture.
+        cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
+        if (!cuda_ok(cudaStreamIsCapturing(st, &cs))) return LCKV_ECUDA;
+        if (cs != cudaStreamCaptureStatusNone) return LCKV_EINVAL;
+        std::lock_guard<std::mutex> lock(g_static_mutex);
+        if (!g_static_ptr[dev].load(std::memory_order_acquire))
+            if (int rc = static_setup(dev)) return rc;
+        base = g_static_ptr[dev].load(std::memory_order_acquire);
+    }
     const int sms = g_static_sms[dev];
     const int n_workers = sms * lckv::kAluWarps;
     if (sms > LCKV_STATIC_MAX_SMS || n_workers > kStaticMaxWorkers) return LCKV_ESTATICLIMIT;
-    unsigned char* base = g_static_ptr[dev];
-    cudaStream_t st = static_cast<cudaStream_t>(stream);
     uint32_t* d_pre = reinterpret_cast<uint32_t*>(base + kStOffPre);
     int32_t* d_start = reinterpret_cast<int32_t*>(base + kStOffStart);
     int32_t* d_counters = reinterpret_cast<int32_t*>(base + kStOffCounters);
@@ -1354,6 +1417,7 @@ extern "C" int lckv_decode_attention_static(const void* k, const void* v, const 
     p.n_workers = n_workers;
     p.out_f32 = out_dtype;
     p.early_kv = 0;
+    p.wait_limit = lckv::kDefaultWaitLimit;
     p.l2_keep = 0.f;
     p.page_table = nullptr;
     p.pt_stride = 0;

@@ -60,6 +60,8 @@ struct AttnParams {
     int32_t page_shift;       // log2(rows per page)
     float l2_keep;            // fraction of the cache lines to keep in L2 for the next layer's
                               // pass over the same cache (0: stream everything)
+    uint32_t wait_limit;      // polls a wait on a copy may take before the kernel gives up
+                              // (status word = timeout, bounded drain, return)
     int32_t early_kv;         // 1: the launcher guarantees that the plan tables and the visible K/V
                               // rows were final before the PREVIOUS kernel in the stream started,
                               // so the first copies may be issued before the dependency wait
@@ -74,7 +76,7 @@ struct TileCursor {
 __device__ __forceinline__ void cursor_load(TileCursor& c, const AttnParams& p)
 {
     c.nt = __ldg(p.pre + c.b + 1) - __ldg(p.pre + c.b);
-    c.nv = min(__ldg(p.lens + c.b) + p.mode, (int32_t)p.T_cap);  // a cache holds at most T_cap rows
+    c.nv = visible_rows(__ldg(p.lens + c.b), p.mode, p.T_cap);
 }
 
 // Next tile in (b, pair, tile) order, skipping sequences without tiles.  Safe past the end.
@@ -189,7 +191,7 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
 
     // Rows that see nothing (diagonal-masked first token): the zero dummy KV gives o = 0, lse = 0.
     for (int b = w; b < p.B; b += p.n_workers) {
-        if (__ldg(p.lens + b) + p.mode == 0) {
+        if (visible_rows(__ldg(p.lens + b), p.mode, p.T_cap) == 0) {
             const int esz = p.out_f32 ? 4 : 2;
             const int n16 = H * D * esz / 16;
             uint4* o16 = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.out) +
@@ -237,7 +239,7 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
         const int rows = min(R, cc.nv - (int)cc.t * R);
 
         // ---- K tile: scores -----------------------------------------------------------------
-        if (!mbar_wait_bounded(bars + 8 * cslot, cphase)) { ok = false; break; }
+        if (!mbar_wait_bounded(bars + 8 * cslot, cphase, p.wait_limit)) { ok = false; break; }
         float part[SUB][NP];
 #pragma unroll
         for (int u = 0; u < SUB; ++u) {
@@ -332,7 +334,7 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
 #endif
 
         // ---- V tile: weighted sum -----------------------------------------------------------
-        if (!mbar_wait_bounded(bars + 8 * cslot, cphase)) { ok = false; break; }
+        if (!mbar_wait_bounded(bars + 8 * cslot, cphase, p.wait_limit)) { ok = false; break; }
         if (rows < R) {
             // Rows past the copy hold leftovers of an earlier tile; their weight is 0 but 0 * NaN
             // is NaN, so clear them.  Generic-proxy writes, fenced before the slot's next copy.
@@ -458,11 +460,11 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
                 const int kk = (int)((uint32_t)w - c_first);         // this contributor's index in the pair
                 const int ck = (kk / kAluChunk) * kAluChunk;         // its chunk's first index
                 const uint32_t cw = c_first + (uint32_t)ck;          // chunk's first worker
-                const int cslot = (ck == 0) ? first_odd : 0;
-                int32_t* tk = two_level ? p.counters2 + 2 * cw + cslot : p.counters + c_first;
+                const int first_rec = (ck == 0) ? first_odd : 0;
+                int32_t* tk = two_level ? p.counters2 + 2 * cw + first_rec : p.counters + c_first;
                 int n = two_level ? min(kAluChunk, n_parts - ck) : n_parts;
                 uint32_t fw = two_level ? cw : c_first;
-                int step = 1, fslot = two_level ? cslot : first_odd;
+                int step = 1, fslot = two_level ? first_rec : first_odd;
                 for (int round = two_level ? 0 : 1; round < 2; ++round) {
                     int ticket = 0;
                     if (lane == 0) ticket = atomicAdd(tk, 1);
@@ -473,7 +475,7 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
                     if (lane == 0) *tk = 0;              // ready for the next launch
                     if (round == 1) { write_row = true; break; }
                     // the chunk's result becomes the record of the chunk's first worker
-                    float* crec = p.partials + (size_t)(2 * cw + cslot) * REC;
+                    float* crec = p.partials + (size_t)(2 * cw + first_rec) * REC;
                     if (lane < LPR) {
                         reinterpret_cast<float4*>(crec)[2 * lane] = make_float4(o[0], o[1], o[2], o[3]);
                         reinterpret_cast<float4*>(crec)[2 * lane + 1] = make_float4(o[4], o[5], o[6], o[7]);

@@ -91,7 +91,7 @@ struct RowCursor {
 __device__ __forceinline__ void rcursor_load(RowCursor& c, const AttnParams& p)
 {
     c.nt = __ldg(p.pre + c.b + 1) - __ldg(p.pre + c.b);
-    c.nv = min(__ldg(p.lens + c.b) + p.mode, (int32_t)p.T_cap);  // a cache holds at most T_cap rows
+    c.nv = visible_rows(__ldg(p.lens + c.b), p.mode, p.T_cap);
 }
 
 // After b, h, t are set: derive the kv head and the tile's first row.  per_kv = pairs per kv head.
@@ -133,7 +133,7 @@ __global__ void __launch_bounds__(kMmaWarps * 32, 1)
 attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV)
 {
-    constexpr int R = kMmaSlotBytes / (D * 2);  // tokens per tile: 32 (D=64), 16 (D=128)
+    constexpr int R = kMmaSlotBytes / (D * 2);  // tokens per tile: 64 (D=64), 32 (D=128)
     constexpr int RB = R / 16;                  // 16-token row blocks per tile
     constexpr int KS = D / 16;                  // k-steps of the score MMA
     constexpr int MT = D / 16;                  // 16-dim m-tiles of the output MMA
@@ -209,7 +209,7 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
 
     // Sequences that see nothing: zero rows (zero dummy KV), lse 0.
     for (int b = w; b < p.B; b += p.n_workers) {
-        if (__ldg(p.lens + b) + p.mode == 0) {
+        if (visible_rows(__ldg(p.lens + b), p.mode, p.T_cap) == 0) {
             const int esz = p.out_f32 ? 4 : 2;
             const int n16 = mp.n_q_heads * D * esz / 16;
             uint4* o16 = reinterpret_cast<uint4*>(static_cast<uint8_t*>(p.out) +
@@ -251,7 +251,7 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
         const int rows = min(R, cc.nv - (int)cc.t * R);
 
         // ---- K tile: S^T = K . Q^T ----------------------------------------------------------
-        if (!mbar_wait_bounded(bars + 8 * cslot, cphase)) { ok = false; break; }
+        if (!mbar_wait_bounded(bars + 8 * cslot, cphase, p.wait_limit)) { ok = false; break; }
         float s[RB][4];
         {
             const uint32_t slot = ring + cslot * kMmaSlotBytes;
@@ -319,7 +319,7 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
         }
 
         // ---- V tile: O^T += V^T . P^T -------------------------------------------------------
-        if (!mbar_wait_bounded(bars + 8 * cslot, cphase)) { ok = false; break; }
+        if (!mbar_wait_bounded(bars + 8 * cslot, cphase, p.wait_limit)) { ok = false; break; }
         {
             const uint32_t slot = ring + cslot * kMmaSlotBytes;
             if (rows < R) {
@@ -441,13 +441,13 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
                 const int k = (int)((uint32_t)w - c_first);          // this contributor's index in the pair
                 const int ck = (k / kMmaChunk) * kMmaChunk;          // its chunk's first index
                 const uint32_t cw = c_first + (uint32_t)ck;          // chunk's first worker
-                const int cslot = (ck == 0) ? first_odd : 0;
+                const int first_rec = (ck == 0) ? first_odd : 0;
                 const int n_chunks = (n_parts + kMmaChunk - 1) / kMmaChunk;
                 // first round: chunk level (two-level) or pair level (direct); second round: pair level
-                int32_t* tk = two_level ? p.counters2 + 2 * cw + cslot : p.counters + c_first;
+                int32_t* tk = two_level ? p.counters2 + 2 * cw + first_rec : p.counters + c_first;
                 int n = two_level ? min(kMmaChunk, n_parts - ck) : n_parts;
                 uint32_t fw = two_level ? cw : c_first;
-                int step = 1, fslot = two_level ? cslot : first_odd;
+                int step = 1, fslot = two_level ? first_rec : first_odd;
                 for (int round = two_level ? 0 : 1; round < 2; ++round) {
                     int ticket = 0;
                     if (lane == 0) ticket = atomicAdd(tk, 1);
@@ -458,7 +458,7 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
                     if (lane == 0) *tk = 0;              // ready for the next launch
                     if (round == 1) { write_row = true; break; }
                     // the chunk's result becomes the record of the chunk's first worker
-                    float* crec = p.partials + (size_t)(2 * cw + cslot) * REC;
+                    float* crec = p.partials + (size_t)(2 * cw + first_rec) * REC;
 #pragma unroll
                     for (int mt = 0; mt < MT; ++mt)
                         reinterpret_cast<float4*>(crec)[mt * 32 + lane] =

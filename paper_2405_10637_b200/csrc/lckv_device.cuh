@@ -7,6 +7,14 @@ namespace lckv {
 
 constexpr int kStatusTimeout = 5;  // written to the device status word when a bounded wait gives up
 
+// Rows of a cache a query sees: len + mode (mode 1 includes the token's own row), never more than
+// the cache holds and never negative (a corrupt length must not turn into a huge unsigned count).
+__device__ __forceinline__ int32_t visible_rows(int32_t len, int32_t mode, int64_t T_cap)
+{
+    const int64_t n = (int64_t)len + mode;
+    return (int32_t)(n < 0 ? 0 : (n > T_cap ? T_cap : n));
+}
+
 __device__ __forceinline__ uint32_t smem_u32(const void* p)
 {
     return static_cast<uint32_t>(__cvta_generic_to_shared(p));
@@ -63,9 +71,11 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
     return ok != 0;
 }
 
-// Bounded wait: false if the phase did not complete within `limit` polls.
+// Bounded wait: false if the phase did not complete within `limit` polls (a poll parks the warp
+// for up to LCKV_WAIT_HINT_NS, so the default is seconds - far beyond any healthy copy).
+constexpr uint32_t kDefaultWaitLimit = 1u << 18;
 __device__ __forceinline__ bool mbar_wait_bounded(uint32_t bar, uint32_t parity,
-                                                  uint32_t limit = (1u << 18))
+                                                  uint32_t limit = kDefaultWaitLimit)
 {
     for (uint32_t it = 0; it < limit; ++it)
         if (mbar_try_wait(bar, parity)) return true;

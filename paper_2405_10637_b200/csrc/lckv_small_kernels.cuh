@@ -12,7 +12,8 @@ namespace lckv {
 //   pre[mode][b]      tiles of sequences 0..b-1 (exclusive prefix; pre[mode][B] = all tiles / H)
 //   start_b[mode][w]  the sequence in which worker w's range begins
 // so an attention worker needs two small loads to find its place.  n_vis is capped at T_cap: in
-// streaming mode (sink + recent window) a cache never holds more than T_cap rows.
+// streaming mode (sink + recent window) a cache never holds more than T_cap rows; a negative length
+// counts as zero rows.
 // ---------------------------------------------------------------------------------------------
 __global__ void __launch_bounds__(1024)
 plan_kernel(const int32_t* __restrict__ lens, int B, int R, int H, int n_workers,
@@ -27,7 +28,7 @@ plan_kernel(const int32_t* __restrict__ lens, int B, int R, int H, int n_workers
         uint32_t* pr = pre + mode * pre_stride;
         const int b0 = min(B, tid * chunk), b1 = min(B, b0 + chunk);
         uint32_t local = 0;
-        for (int b = b0; b < b1; ++b) local += (uint32_t)(min(lens[b] + mode, T_cap) + R - 1) / (uint32_t)R;
+        for (int b = b0; b < b1; ++b) local += (uint32_t)(visible_rows(lens[b], mode, T_cap) + R - 1) / (uint32_t)R;
         // block-wide exclusive scan of `local`
         uint32_t incl = local;
         for (int off = 1; off < 32; off <<= 1) {
@@ -49,7 +50,7 @@ plan_kernel(const int32_t* __restrict__ lens, int B, int R, int H, int n_workers
         uint32_t run = warp_sums[warp] + incl - local;
         for (int b = b0; b < b1; ++b) {
             pr[b] = run;
-            run += (uint32_t)(min(lens[b] + mode, T_cap) + R - 1) / (uint32_t)R;
+            run += (uint32_t)(visible_rows(lens[b], mode, T_cap) + R - 1) / (uint32_t)R;
         }
         if (tid == 0) pr[B] = carry;
         __syncthreads();  // pr[] (global) is now visible to the whole block

@@ -11,25 +11,33 @@ REL_L2 = 5e-3      # tolerance on ||gpu - oracle||_2 / ||oracle||_2
 NAN_BITS = 0x7FC0  # bf16 quiet NaN, used to poison rows that must never be read
 
 
+def bf16_tolerance(want):
+    """Per-element bound on |gpu - oracle| for a bf16 output: MAX_ABS, except where the value is so
+    large that one rounding to bf16 alone can exceed it.  In the binade [4, 8) half an ulp is 2^-6 =
+    0.0156 > MAX_ABS (below 4 it is at most 0.0078, so the plain bound is attainable there); such
+    elements - they occur with N(0,1) values at contexts of a few tokens - get 2^-8 |o|, between half
+    an ulp and one ulp of their binade."""
+    a = np.abs(want)
+    return np.where(a >= 4.0, a * 2.0 ** -8, MAX_ABS)
+
+
 def compare(got, want, what=""):
-    """got: torch tensor (bf16/fp32) from the GPU; want: float64 numpy from the oracle."""
+    """got: torch tensor (bf16/fp32) from the GPU; want: float64 numpy from the oracle.
+    Returns the observed (max-abs, rel-L2), as measured."""
     g = got.detach().float().cpu().numpy().astype(np.float64)
     assert g.shape == want.shape, (g.shape, want.shape)
     assert np.isfinite(g).all(), f"{what}: non-finite GPU output"
     zero_rows = ~want.any(axis=-1)
     assert not g[zero_rows].any(), f"{what}: rows the oracle gives as exactly 0 are not 0"
     err = np.abs(g - want)
-    max_abs = err.max() if g.size else 0.0
-    if got.dtype == torch.bfloat16:
-        # A bf16 output cannot be closer than half an ulp (2^-9 relative) to the true value, which
-        # exceeds 1e-2 once |o| > 5.12 and comes close to it from |o| = 4 on (short contexts with
-        # N(0,1) values do reach that).  Elements that large are allowed one bf16 ulp instead.
-        excess = err - np.maximum(MAX_ABS, np.abs(want) * 2.0 ** -8)
-        assert excess.max() <= 0, f"{what}: max-abs {max_abs:.3e} beyond tolerance and bf16 ulp"
-        max_abs = min(max_abs, MAX_ABS) if excess.max() <= 0 else max_abs
+    max_abs = float(err.max()) if g.size else 0.0
+    tol = bf16_tolerance(want) if got.dtype == torch.bfloat16 else MAX_ABS
+    excess = err - tol
+    if g.size:
+        i = np.unravel_index(np.argmax(excess), excess.shape)
+        assert excess[i] <= 0, f"{what}: |gpu - oracle| = {err[i]:.3e} at {i} (oracle {want[i]:.4f})"
     denom = np.linalg.norm(want[~zero_rows])
-    rel = np.linalg.norm((g - want)[~zero_rows]) / denom if denom > 0 else 0.0
-    assert max_abs <= MAX_ABS, f"{what}: max-abs {max_abs:.3e}"
+    rel = float(np.linalg.norm((g - want)[~zero_rows]) / denom) if denom > 0 else 0.0
     assert rel <= REL_L2, f"{what}: rel-L2 {rel:.3e}"
     return max_abs, rel
 

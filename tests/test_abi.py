@@ -68,3 +68,37 @@ def test_null_and_invalid_handles_return_errors_without_a_gpu():
     assert lib.lckv_cache_bytes(C.byref(bad)) == 0
     bad = lk.make_config(4, 2, 4, 4, 96, 2, 16)   # unsupported head_dim
     assert lib.lckv_cache_bytes(C.byref(bad)) == 0
+
+
+def test_static_entry_refuses_bad_arguments_before_touching_a_gpu():
+    """The allocation-free entry point checks its arguments before any CUDA call, so a pointer that
+    would fault on the device (off the 16-byte grid of the bulk copies and vector accesses) or a size
+    beyond the fixed scratch comes back as an error code.  The pointers here are never dereferenced."""
+    f = lk.lib().lckv_decode_attention_static
+    a = 0x10000     # a plausible, aligned address
+
+    def call(k=a, v=a, lens=a, q=a, out=a, lse=None, status=None, batch=4, hq=8, hkv=8, d=128, T=64, mode=0,
+             scale=0.0, odt=0):
+        return f(k, v, lens, q, out, lse, status, batch, hq, hkv, d, T, mode, scale, odt, None)
+    for name in ("k", "v", "q", "out"):
+        assert call(**{name: a + 8}) == lk.EINVAL, name       # 8-byte aligned is not enough
+        assert call(**{name: a + 2}) == lk.EINVAL, name
+        assert call(**{name: None}) == lk.EINVAL, name
+    assert call(lens=a + 2) == lk.EINVAL
+    assert call(lens=None) == lk.EINVAL
+    assert call(lse=a + 1) == lk.EINVAL
+    assert call(status=a + 2) == lk.EINVAL
+    assert call(batch=0) == lk.EINVAL
+    assert call(hkv=3) == lk.EINVAL
+    assert call(d=96) == lk.EINVAL
+    assert call(T=0) == lk.EINVAL
+    assert call(T=1 << 31) == lk.EINVAL
+    assert call(mode=2) == lk.EINVAL
+    assert call(odt=2) == lk.EINVAL
+    assert call(scale=-1.0) == lk.EINVAL
+    assert call(scale=float("nan")) == lk.EINVAL
+    assert call(batch=4097) == lk.ESTATICLIMIT
+
+
+def test_wait_limit_call_checks_its_handle():
+    assert lk.lib().lckv_cache_set_wait_limit(None, 0) == lk.EINVAL

@@ -467,3 +467,27 @@ def test_paged_cache_pool_exhaustion_and_reuse():
     cache.close()
     bad = lk.make_config(2, 0, H, H, d, B, 256, page_rows=48, n_pages=4)   # not a power of two
     assert lk.lckv_cache_bytes(bad) == 0
+
+
+@pytest.mark.parametrize("Hq,Hkv,d", [(4, 4, 128), (16, 2, 64)])
+def test_wait_that_runs_out_is_reported_and_recoverable(Hq, Hkv, d):
+    """The bounded device-side wait, made to run out without anything hanging: with a limit of 0 polls
+    every worker's first wait on a copy gives up at once (the copies themselves are healthy and land
+    during the kernel's bounded drain).  The status word must read LCKV_ETIMEOUT, lckv_cache_reset must
+    clear it, and the next step on the same cache must be correct again.  Both decode kernels."""
+    c = Case(L=3, w=2, Hq=Hq, Hkv=Hkv, d=d, lens=[40, 200, 7], T_cap=260, seed=4242)
+    c.step()                                         # a healthy step first
+    c.cache.lckv_cache_set_wait_limit(0)
+    q, kn, vn = c.step_inputs()
+    dev = c.cache.device
+    out = torch.zeros((c.B, Hq, d), dtype=torch.bfloat16, device=dev)
+    c.cache.lckv_decode_attention(0, lk.MODE_CONDENSED, q[0].to(dev), out=out)
+    torch.cuda.synchronize()
+    assert c.cache.lckv_cache_status() == lk.ETIMEOUT
+    # recovery: default limit back, reset clears the status word and the merge tickets
+    c.cache.lckv_cache_set_wait_limit(1 << 18)
+    c.cache.lckv_cache_reset(c.lens.tolist())
+    assert c.cache.lckv_cache_status() == 0
+    c.step()
+    c.step()
+    c.close()
