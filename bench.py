@@ -34,32 +34,52 @@ METRIC = "condensed decode-attn GB/s (% of 8 TB/s HBM) and layer-stack attn µs/
 NOMINAL_HBM_GBS = 8000.0
 
 
-# DRAM counters of one captured launch per kernel (ncu, small case; summaries under profiles/).  Reads grow
-# with the rows read, so they are scaled by the algorithmic input bytes; the writes beyond the output rows
-# (split-K partials, bounded by the worker count, and write-backs) are a per-launch constant.
-NCU_CAPTURES = {
-    "attn_alu_kernel": {
-        "source": "profiles/attn_alu_kernel_llama7b_b8_ncu_full.md",
-        "alg_in": 283.9e6 - 65536, "read": 284.00e6, "write": 3.46e6, "out": 65536,
-        "applies": lambda a: a.workload in ("llama7b", "llama30b", "sweep7b") and not a.page_rows,
-    },
-    "attn_mma_kernel": {
-        "source": "profiles/attn_mma_kernel_tinyllama_b128_ncu_full.md",
-        "alg_in": 135.3e6 - 524288, "read": 143.21e6, "write": 4.6e6, "out": 524288,
-        # the over-read of whole 64-row boxes depends on where the lengths sit: default context only
-        "applies": lambda a: a.workload == "tinyllama" and a.context in (0, 1024) and a.batch in (0, 128)
-        and not a.page_rows,
-    },
-}
+# DRAM counters of one captured launch per kernel (ncu, small case): profiles/ncu_captures.json, written
+# from the summaries beside it.  Reads grow with the rows read, so they are scaled by the algorithmic
+# input bytes; the writes beyond the output rows (split-K partials, bounded by the worker count, and
+# write-backs) are a per-launch constant.  A capture is void once the kernel's sources differ from
+# the ones it was taken with (digest of the files named in the entry).
+CAPTURES_FILE = os.path.join(ROOT, "profiles", "ncu_captures.json")
+CSRC = os.path.join(ROOT, "paper_2405_10637_b200", "csrc")
 
 
-def scaled_traffic(kernel, args, alg_bytes, out_bytes):
-    """dram read + write bytes of one launch, scaled from the captured launch; None where it does not apply."""
-    cap = NCU_CAPTURES[kernel]
-    if not cap["applies"](args):
+def source_digest(files):
+    """sha256 over the named kernel sources, in order."""
+    import hashlib
+    h = hashlib.sha256()
+    for f in files:
+        with open(os.path.join(CSRC, f), "rb") as fh:
+            h.update(fh.read())
+    return h.hexdigest()[:16]
+
+
+def load_captures():
+    with open(CAPTURES_FILE) as f:
+        return json.load(f)
+
+
+def capture_applies(cap, args):
+    """Does the captured launch's traffic scale to this run's launches?"""
+    c = cap["applies"]
+    if args.workload not in c["workloads"] or args.page_rows or args.stream_sink:
+        return False
+    if "contexts" in c and args.context not in c["contexts"]:
+        return False
+    if "batches" in c and args.batch not in c["batches"]:
+        return False
+    return True
+
+
+def scaled_traffic(kernel, args, alg_bytes, out_bytes, captures=None, check_sources=True):
+    """dram read + write bytes of one launch, scaled from the captured launch; None where the capture
+    does not apply or the kernel has changed since."""
+    cap = (captures or load_captures()).get(kernel)
+    if cap is None or not capture_applies(cap, args):
         return None
-    reads = cap["read"] / cap["alg_in"] * (alg_bytes - out_bytes)
-    return reads + out_bytes + (cap["write"] - cap["out"])
+    if check_sources and source_digest(cap["sources"]) != cap["sources_digest"]:
+        return None
+    reads = cap["dram_read_bytes"] / cap["algorithmic_input_bytes"] * (alg_bytes - out_bytes)
+    return reads + out_bytes + (cap["dram_write_bytes"] - cap["output_bytes"])
 
 
 def measured_peaks():
@@ -256,6 +276,118 @@ def time_steps(fn, steps, stream):
     return e0.elapsed_time(e1)
 
 
+def bf16_peak():
+    try:
+        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
+            return float(json.load(fh)["bf16_tflops"]), "measured"
+    except Exception:
+        return 1590.0, "fallback"
+
+
+def fill_cache(cache, wl, rank=0, seqs=None):
+    """Seeded N(0, std) keys and values in every slot.  seqs = (b0, b1): this cache holds sequences
+    [b0, b1) of one global batch and each sequence is drawn from its own seed, so the shards of a batch
+    hold the same bits however many ranks share it."""
+    for s in range(cache.info.n_slots):
+        kt, vt = cache.slot_tensors(s)
+        if seqs is None:
+            syn.fill_randn_bf16_(kt, syn.seed_for(wl, syn.T_K, s + 16 * rank), std=wl.std)
+            syn.fill_randn_bf16_(vt, syn.seed_for(wl, syn.T_V, s + 16 * rank), std=wl.std)
+        else:
+            for i, b in enumerate(range(*seqs)):
+                syn.fill_randn_bf16_(kt[i], syn.seed_for(wl, syn.T_K, 64 * (b + 1) + s), std=wl.std)
+                syn.fill_randn_bf16_(vt[i], syn.seed_for(wl, syn.T_V, 64 * (b + 1) + s), std=wl.std)
+
+
+def read_stream_probe(lk, buf, stream, nbytes=8 << 30):
+    """Read-only stream over the first `nbytes` of a device buffer with the library's probe kernels:
+    GB/s per kind (best of 5 after 2 warm-up passes) - the ceiling of a read-dominated kernel."""
+    nbytes = min(nbytes, buf.numel() * buf.element_size()) // 8192 * 8192
+    acc = torch.zeros(1, dtype=torch.int32, device=buf.device)
+    status = torch.zeros(1, dtype=torch.int32, device=buf.device)
+    out = {"bytes": nbytes}
+    for kind, name in ((0, "ldg16"), (2, "ldg32"), (1, "bulk8k")):
+        def f():
+            lk.lckv_read_stream_probe(buf, nbytes, kind, acc, status)
+        for _ in range(2):
+            f()
+        torch.cuda.synchronize()
+        best = min(time_steps(f, 1, stream) for _ in range(5))
+        out[name] = nbytes / (best * 1e-3) / 1e9
+    assert int(status.item()) == 0, "probe wait timed out"
+    out["best"] = max(out["ldg16"], out["ldg32"], out["bulk8k"])
+    return out
+
+
+def time_workload(lk, dev, stream, wl, B, lens, T_cap, steps, warm=3, graph=1, top_variant=0):
+    """Allocates the caches of one workload, fills them, times `steps` decode steps (after `warm`),
+    frees everything.  Returns the compact record used in the `configs` array."""
+    L = wl.n_layers
+    cfg = lk.make_config(L, wl.n_warmup, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, B, T_cap,
+                         use_graph=graph, top_variant=top_variant)
+    cache = lk.Cache(cfg, device=dev)
+    try:
+        plan = lk.lckv_plan(L, wl.n_warmup, top_variant)
+        fill_cache(cache, wl)
+        q = [syn.randn_bf16((B, wl.n_q_heads, wl.head_dim), 900 + l, device=dev, std=wl.std) for l in range(L)]
+        kv = [syn.randn_bf16((B, wl.n_kv_heads, wl.head_dim), 950 + l, device=dev, std=wl.std)
+              if plan["write_slot"][l] >= 0 else None for l in range(L)]
+        outs = [torch.empty((B, wl.n_q_heads, wl.head_dim), dtype=torch.bfloat16, device=dev) for _ in range(L)]
+        cache.lckv_cache_reset(np.asarray(lens).tolist(), batch=B)
+
+        def f():
+            cache.lckv_layer_stack_step(q, outs, kv, kv, batch=B)
+        for _ in range(warm):
+            f()
+        torch.cuda.synchronize()
+        ms = time_steps(f, steps, stream) / steps
+        by = sum(step_kv_bytes(wl, plan["mode"], lens, B, warm + i) for i in range(steps)) / steps
+        assert cache.lckv_cache_status() == 0, "device-side wait timed out"
+        info = cache.info
+        gbs = by / (ms * 1e-3) / 1e9
+        return {"us_per_step": ms * 1e3, "kv_GBps": gbs, "frac_of_8TBs": gbs / NOMINAL_HBM_GBS,
+                "kv_bytes_per_step": by, "cache_bytes": int(2 * info.n_slots * info.slot_bytes),
+                "footprint_slots": info.n_slots, "B": B, "steps": steps,
+                "kernel": "attn_alu_kernel" if info.kernel_kind == 1 else "attn_mma_kernel"}
+    finally:
+        cache.close()
+        del cache
+        torch.cuda.empty_cache()
+
+
+def largest_batch(wl, T_cap, n_slots, budget_bytes=180e9):
+    """Largest batch whose caches (n_slots of them, T_cap rows per sequence) fit the budget."""
+    return int(budget_bytes // (n_slots * 4 * wl.n_kv_heads * wl.head_dim * T_cap))
+
+
+def config_matrix(lk, dev, stream):
+    """The other workload shapes, each a few decode steps: toy, TinyLlama (B = 128 at three context
+    lengths of the 512 + 1024 run), the 30B shape at the largest batch that fits, and the warmup-count
+    sweep on the 7B shape at both long-context sizes."""
+    W = syn.WORKLOADS
+    rows = []
+
+    def add(name, wl, B, T, steps, T_cap=None, **kw):
+        r = time_workload(lk, dev, stream, wl, B, np.full(B, T, np.int32), T_cap or T + steps + 8, steps, **kw)
+        r["workload"] = name
+        rows.append(r)
+    add("toy L4 MHA4 d64 w0 B2 T128", W["toy"], 2, 128, 50)
+    for T in (512, 1024, 1535):   # start, middle and end of the 512 + 1024 run
+        add(f"tinyllama B128 T{T}", W["tinyllama"], 128, T, 30)
+    # 30B shape: 2 caches (w = 2, literal reading of "top layer"), 4096 rows per sequence
+    free = torch.cuda.mem_get_info()[0]
+    wl = W["llama30b"]
+    B30 = min(largest_batch(wl, 4096, 2), largest_batch(wl, 4096, 2, free - 6e9))
+    add(f"llama30b w2 B{B30} T2048 (largest batch whose caches fit 180 GB)", wl, B30, 2048, 3, T_cap=4096)
+    for w in (0, 2, 4, 8, 32):
+        wl = W["sweep7b"].with_(n_warmup=w)
+        B = 64 if w < 32 else min(40, largest_batch(wl, 8192 + 16, 32, free - 6e9))   # 64 sequences x 32 caches = 275 GB: does not fit
+        add(f"sweep7b w{w} B{B} T8192", wl, B, 8192, 4)
+    for w in (0, 2, 32):
+        add(f"sweep7b w{w} B8 T32768", W["sweep7b"].with_(n_warmup=w), 8, 32768, 4)
+    return rows
+
+
 def run_ours(args):
     from paper_2405_10637_b200 import binding as lk
     rank = int(os.environ.get("RANK", "0"))
@@ -273,15 +405,26 @@ def run_ours(args):
     stream = torch.cuda.current_stream()
 
     wl, p = workload_params(args)
-    B, T_cap = p["batch"], p["t_cap"]
     L = wl.n_layers
-    # every rank draws its own sequences (different seeds): independent replicas of the workload
-    lens = syn.ragged_lengths(B, p["lo"], p["hi"], syn.seed_for(wl, syn.T_LENS, rank)).numpy()
+    B_job, T_cap = p["batch"], p["t_cap"]
+    # Sharding.  Default: every rank runs the whole per-GPU workload on sequences of its own
+    # (replicas, weak scaling).  --shard batch / heads: ONE seeded batch of B_job sequences is split
+    # over the ranks by sequences or by kv heads (strong scaling); no rank needs another's data.
+    b0, b1, h0, h1 = 0, B_job, 0, wl.n_kv_heads
+    if args.shard == "batch":
+        b0, b1 = syn.shard_batch(B_job, rank, world)
+    elif args.shard == "heads":
+        h0, h1 = syn.shard_heads(wl.n_kv_heads, rank, world)
+    B = b1 - b0
+    g = wl.n_q_heads // wl.n_kv_heads
+    wl_local = wl.with_(n_q_heads=(h1 - h0) * g, n_kv_heads=h1 - h0)
+    lens_seed = syn.seed_for(wl, syn.T_LENS, 0 if args.shard else rank)
+    lens = syn.ragged_lengths(B_job, p["lo"], p["hi"], lens_seed).numpy()[b0:b1]
     n_pages = 0
     if args.page_rows:   # pool: what the sequences hold at the end of the longest timed run, + 2 %
         grow = max(64, args.steps + args.warmup + 8)
         n_pages = int(1.02 * sum((int(x) + grow + args.page_rows - 1) // args.page_rows for x in lens)) + 8
-    cfg = lk.make_config(L, wl.n_warmup, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, B, T_cap,
+    cfg = lk.make_config(L, wl.n_warmup, wl_local.n_q_heads, wl_local.n_kv_heads, wl.head_dim, B, T_cap,
                          host_staging=1, use_graph=1 if args.graph else 0, kernel_kind=args.kernel_kind,
                          top_variant=args.top_variant, stream_sink=args.stream_sink,
                          page_rows=args.page_rows, n_pages=n_pages)
@@ -289,10 +432,11 @@ def run_ours(args):
     cache = lk.Cache(cfg, device=dev)
     plan = lk.lckv_plan(L, wl.n_warmup, args.top_variant)
     info = cache.info
-    for s in range(info.n_slots):
-        kt, vt = cache.slot_tensors(s)
-        syn.fill_randn_bf16_(kt, syn.seed_for(wl, syn.T_K, s + 16 * rank), std=wl.std)
-        syn.fill_randn_bf16_(vt, syn.seed_for(wl, syn.T_V, s + 16 * rank), std=wl.std)
+    if args.shard:
+        fill_sharded(cache, wl, b0, b1, h0, h1)
+    else:
+        fill_cache(cache, wl, rank)
+    wl = wl_local
     q = [syn.randn_bf16((B, wl.n_q_heads, wl.head_dim), 900 + l, device=dev, std=wl.std)
          for l in range(L)]
     kv = [syn.randn_bf16((B, wl.n_kv_heads, wl.head_dim), 950 + l, device=dev, std=wl.std)
@@ -342,7 +486,8 @@ def run_ours(args):
     barrier()
     clocks = sampler.stop() if rank == 0 else None
     ms_step = max_over_ranks(ms_step)
-    value = world * bytes_step / (ms_step * 1e-3) / 1e9
+    # whole-job bytes: all ranks' units over the slowest rank's time
+    value = multi.sum_over_ranks(bytes_step, dev) / (ms_step * 1e-3) / 1e9
     assert cache.lckv_cache_status() == 0, "device-side wait timed out"
 
     # ---- roofline of the dominant kernel: condensed attention launches on the shared cache ------
@@ -361,17 +506,24 @@ def run_ours(args):
     peak, peak_kind = measured_peaks()
     achieved = alg_bytes / (ms_attn * 1e-3) / 1e9
     kernel_name = "attn_alu_kernel" if info.kernel_kind == 1 else "attn_mma_kernel"
-    traffic = scaled_traffic(kernel_name, args, alg_bytes, io_bytes // 2)
+    captures = load_captures()
+    traffic = None if args.shard else scaled_traffic(kernel_name, args, alg_bytes, io_bytes // 2, captures)
+    probe = read_stream_probe(lk, cache.buf, stream)
     roofline = {"bound": "hbm", "achieved": achieved, "peak": peak, "unit": "GB/s",
                 "frac": achieved / peak, "traffic": traffic, "peak_kind": peak_kind,
+                "peak_note": "the measured peak is a read + write copy; a read-only stream on this GPU "
+                             "reaches read_stream_gbs (this library's probe kernels, "
+                             f"{probe['bytes'] >> 30} GiB), which is the ceiling of this read-dominated kernel",
+                "read_stream_gbs": probe["best"], "read_stream": probe,
+                "frac_of_read_stream": achieved / probe["best"],
                 "kernel": kernel_name,
-                "traffic_source": NCU_CAPTURES[kernel_name]["source"] if traffic else None,
+                "traffic_source": captures[kernel_name]["source"] if traffic else None,
                 "us_per_launch": ms_attn * 1e3, "algorithmic_bytes_per_launch": alg_bytes,
                 "frac_of_nominal_8TBs": achieved / NOMINAL_HBM_GBS}
 
     # ---- batch sweep (µs/step vs B) ---------------------------------------------------------
     sweep = []
-    for b in p["sweep"]:
+    for b in ([] if args.shard else p["sweep"]):
         if b > B:
             continue
         f = make_step(b)
@@ -401,7 +553,7 @@ def run_ours(args):
     ms_e2e = max_over_ranks(ms_e2e)
     h2d = sum(t.numel() * 2 for t in hq) + 2 * sum(t.numel() * 2 for t in hkv if t is not None)
     d2h = sum(t.numel() * 2 for t in hout)
-    e2e = {"value": world * by_e2e / (ms_e2e * 1e-3) / 1e9, "unit": "GB/s",
+    e2e = {"value": multi.sum_over_ranks(by_e2e, dev) / (ms_e2e * 1e-3) / 1e9, "unit": "GB/s",
            "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e}
 
     # ---- CPU baseline: the checker on a bounded sample (rank 0, N = 1 only) --------------------
@@ -416,37 +568,77 @@ def run_ours(args):
         cpu = {"value": gbs, "unit": "GB/s", "cores": cores, "kind": "oracle",
                "sample": f"first {rows} of {B} sequences, all {L} layers, {n} repetitions of one "
                          f"decode step ({sec:.2f} s each)"}
+        del Ks, Vs
+
+    launches = info.launches_per_step * args.steps
+    cache_bytes = int(2 * info.n_slots * info.slot_bytes)
+    slots = info.n_slots
+    cache.close()
+    del cache, hq_all, hkv_all, hout_all
+    torch.cuda.empty_cache()
+
+    # ---- the other workload shapes and the kernels beside the decode path (N = 1, default run) ---
+    configs = nxt = clocks_extras = None
+    if world == 1 and args.extras:
+        sampler = ClockSampler(local)
+        sampler.start()
+        configs = config_matrix(lk, dev, stream)
+        nxt = {"prompt_encoding_n8192": prefill_record(lk, dev, W7B(), 8192, 8, 10),
+               "kv_producer_b16": project_record(lk, dev, W7B(), 4096, 16, 20),
+               "kv_producer_b512": project_record(lk, dev, W7B(), 4096, 512, 20)}
+        clocks_extras = sampler.stop()
 
     if rank == 0:
+        layer_pass_bytes = bytes_step / L
         print(json.dumps({
             "metric": METRIC, "value": value, "unit": "GB/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": ms_step, "higher_is_better": True,
-            "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
-            "config": {"workload": workload_name(wl, p), "l2": "inputs larger than L2"
-                       if 2 * info.slot_bytes > 2 * 126e6 else "L2-resident cache: warm",
-                       "kv_bytes_per_step": bytes_step, "footprint_slots": info.n_slots,
+            "scaling": "strong" if args.shard else "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": workload_name(syn.WORKLOADS[args.workload] if args.warmup_layers is None else
+                                                 syn.WORKLOADS[args.workload].with_(n_warmup=args.warmup_layers), p),
+                       "storage_dtype": "bf16 (q, K, V, outputs); fp32 scores, sums, accumulators, partials",
+                       "l2": "inputs larger than L2: a layer's pass over its cache reads "
+                             f"{layer_pass_bytes / 1e6:.0f} MB" if layer_pass_bytes > 2 * 126e6 else
+                             f"a layer's pass reads {layer_pass_bytes / 1e6:.0f} MB, within reach of the 126 MB L2: "
+                             "warm (consecutive layers re-read the shared cache)",
+                       "shard": args.shard or "replicas", "sequences_this_rank": B,
+                       "kv_heads_this_rank": wl.n_kv_heads,
+                       "kv_bytes_per_step": bytes_step, "footprint_slots": slots,
                        "top_variant": args.top_variant, "graph": bool(args.graph),
                        "stream_sink": args.stream_sink, "page_rows": args.page_rows,
-                       "cache_bytes": int(2 * info.n_slots * info.slot_bytes)},
+                       "cache_bytes": cache_bytes},
             "frac_of_8TBs": value / world / NOMINAL_HBM_GBS,
-            "clocks": clocks, "e2e": e2e, "gpu_launches": info.launches_per_step * args.steps,
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
             "roofline": roofline, "cpu_baseline": cpu, "sweep": sweep,
+            "configs": configs, "next": nxt, "clocks_extras": clocks_extras,
         }))
-    cache.close()
     if world > 1:
         import torch.distributed as dist
         dist.destroy_process_group()
 
 
-def run_prefill(args):
-    """--prefill N: times the prompt-encoding attention (one layer, condensed mode, N prompt tokens
-    per sequence) and reports tensor-core throughput.  Not the headline metric: a side measurement."""
-    from paper_2405_10637_b200 import binding as lk
-    wl, p = workload_params(args)
-    n = args.prefill
-    B = args.batch or 8
-    dev = torch.device("cuda:0")
-    torch.cuda.set_device(dev)
+def W7B():
+    return syn.WORKLOADS["llama7b"]
+
+
+def fill_sharded(cache, wl, b0, b1, h0, h1):
+    """Caches of the shard [b0, b1) x kv heads [h0, h1) of one global batch: every (sequence, slot) is
+    drawn from its own seed over ALL kv heads and the shard's heads are copied out, so the shards of
+    any split hold the same bits as the unsplit batch."""
+    for s in range(cache.info.n_slots):
+        kt, vt = cache.slot_tensors(s)
+        full = torch.empty((wl.n_kv_heads,) + tuple(kt.shape[2:]), dtype=torch.bfloat16, device=kt.device)
+        for i, b in enumerate(range(b0, b1)):
+            syn.fill_randn_bf16_(full, syn.seed_for(wl, syn.T_K, 64 * (b + 1) + s), std=wl.std)
+            kt[i].copy_(full[h0:h1])
+            syn.fill_randn_bf16_(full, syn.seed_for(wl, syn.T_V, 64 * (b + 1) + s), std=wl.std)
+            vt[i].copy_(full[h0:h1])
+
+
+def prefill_record(lk, dev, wl, n, B, steps, warm=3):
+    """Prompt-encoding attention (one layer, condensed mask, n prompt tokens per sequence): useful
+    causal TFLOP/s against the measured bf16 peak."""
     cfg = lk.make_config(2, 0, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, B, n)
     cache = lk.Cache(cfg, device=dev)
     kt, vt = cache.slot_tensors(0)
@@ -458,39 +650,44 @@ def run_prefill(args):
 
     def f():
         cache.lckv_prefill_attention(0, lk.MODE_CONDENSED, q, out=out)
-    for _ in range(max(3, args.warmup)):
+    for _ in range(max(3, warm)):
         f()
     torch.cuda.synchronize()
-    ms = time_steps(f, args.steps, stream) / args.steps
+    ms = time_steps(f, steps, stream) / steps
+    assert cache.lckv_cache_status() == 0, "device-side wait timed out"
     # visible (i, j) pairs with j < i: n(n-1)/2 per (sequence, head); 4*d flops per pair (QK^T and PV)
     flops = 4.0 * wl.head_dim * wl.n_q_heads * B * (n * (n - 1) / 2)
-    try:
-        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
-            peak, kind = float(json.load(fh)["bf16_tflops"]), "measured"
-    except Exception:
-        peak, kind = 1590.0, "fallback"
+    peak, kind = bf16_peak()
     tf = flops / (ms * 1e-3) / 1e12
-    print(json.dumps({
-        "metric": "prompt-encoding attention TFLOP/s (causal, useful flops only)", "value": tf,
-        "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
-        "ms_per_step": ms, "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{wl.name} head layout, prompt {n}, B={B}, one layer, j<i mask"},
-        "roofline": {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s",
-                     "frac": tf / peak, "traffic": None, "peak_kind": kind,
-                     "kernel": "prefill_attn_kernel" if os.environ.get("LCKV_PREFILL_KERNEL") == "mma" else "prefill_tc5_kernel"}}))
     cache.close()
+    del cache, q, out
+    torch.cuda.empty_cache()
+    return {"workload": f"{wl.name} head layout, prompt {n}, B={B}, one layer, j<i mask", "ms": ms,
+            "bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
+            "traffic": None, "peak_kind": kind,
+            "kernel": "prefill_attn_kernel" if os.environ.get("LCKV_PREFILL_KERNEL") == "mma" else "prefill_tc5_kernel"}
 
 
-def run_project(args):
-    """--project D: times the fused key/value producer (x W_K^T, x W_V^T -> cache rows) for hidden width
-    D at the workload's head layout.  Several weight sets are used in turn so that their bytes exceed
-    the L2 (as the layers of a model would).  A side measurement, not the headline metric."""
+def run_prefill(args):
+    """--prefill N: times the prompt-encoding attention and reports tensor-core throughput.  Not the
+    headline metric: a side measurement."""
     from paper_2405_10637_b200 import binding as lk
     wl, p = workload_params(args)
-    dm = args.project
-    B = args.batch or 64
     dev = torch.device("cuda:0")
     torch.cuda.set_device(dev)
+    r = prefill_record(lk, dev, wl, args.prefill, args.batch or 8, args.steps, args.warmup)
+    print(json.dumps({
+        "metric": "prompt-encoding attention TFLOP/s (causal, useful flops only)", "value": r["achieved"],
+        "unit": "TFLOP/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+        "ms_per_step": r["ms"], "higher_is_better": True, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": r["workload"]},
+        "roofline": {k: r[k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic", "peak_kind", "kernel")}}))
+
+
+def project_record(lk, dev, wl, dm, B, steps, warm=3):
+    """The fused key/value producer (x W_K^T, x W_V^T -> cache rows) for hidden width dm at the
+    workload's head layout.  Several weight sets are used in turn so that their bytes exceed the L2 (as
+    the layers of a model would)."""
     F = wl.n_kv_heads * wl.head_dim
     T_cap = 64
     cfg = lk.make_config(2, 0, wl.n_q_heads, wl.n_kv_heads, wl.head_dim, B, T_cap)
@@ -512,7 +709,7 @@ def run_project(args):
         i = it[0] % n_sets
         it[0] += 1
         cache.lckv_project_append_kv(0, x, wk[i], wv[i], cos, sin, advance_len=0)
-    for _ in range(max(3, args.warmup) + n_sets):
+    for _ in range(max(3, warm) + n_sets):
         f()
     torch.cuda.synchronize()
     # One call is 10-50 us of device time, less than a Python call costs on the host: replay a captured
@@ -527,31 +724,40 @@ def run_project(args):
     for _ in range(3):
         graph.replay()
     torch.cuda.synchronize()
-    ms = time_steps(graph.replay, args.steps, stream) / (args.steps * n_sets)
+    ms = time_steps(graph.replay, steps, stream) / (steps * n_sets)
     assert cache.lckv_cache_status() == 0, "device-side wait timed out"
     flops = 2.0 * B * 2 * F * dm
     byts = w_bytes + B * dm * 2 + 2 * B * F * 2
-    try:
-        with open(os.path.join(ROOT, "MEASURED_PEAKS.json")) as fh:
-            pk = json.load(fh)
-            peak_tf, peak_gb, kind = float(pk["bf16_tflops"]), float(pk["hbm_gbs"]), "measured"
-    except Exception:
-        peak_tf, peak_gb, kind = 1590.0, 6650.0, "fallback"
+    peak_tf, kind = bf16_peak()
+    peak_gb, _ = measured_peaks()
     tf = flops / (ms * 1e-3) / 1e12
     gbs = byts / (ms * 1e-3) / 1e9
     hbm_bound = byts / peak_gb / 1e9 >= flops / peak_tf / 1e12
     roof = {"bound": "hbm", "achieved": gbs, "peak": peak_gb, "unit": "GB/s", "frac": gbs / peak_gb} if hbm_bound \
         else {"bound": "tensor", "achieved": tf, "peak": peak_tf, "unit": "TFLOP/s", "frac": tf / peak_tf}
     roof.update({"traffic": None, "peak_kind": kind, "kernel": "project_kv_kernel", "tflops": tf, "GBps": gbs,
-                 "algorithmic_bytes_per_launch": byts, "us_per_launch": ms * 1e3})
-    print(json.dumps({
-        "metric": "key/value producer (projection + rotary + append) us per call", "value": ms * 1e3,
-        "unit": "us", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms,
-        "higher_is_better": False, "dtype": "bf16", "data": "synthetic",
-        "config": {"workload": f"{wl.name} head layout, d_model {dm}, B={B}, {n_sets} weight sets in turn",
-                   "l2": "weight sets in rotation exceed L2"},
-        "roofline": roof}))
+                 "algorithmic_bytes_per_launch": byts, "us_per_launch": ms * 1e3,
+                 "workload": f"{wl.name} head layout, d_model {dm}, B={B}, {n_sets} weight sets in turn"})
+    del graph
     cache.close()
+    del cache, wk, wv
+    torch.cuda.empty_cache()
+    return roof
+
+
+def run_project(args):
+    """--project D: times the fused key/value producer.  A side measurement, not the headline metric."""
+    from paper_2405_10637_b200 import binding as lk
+    wl, p = workload_params(args)
+    dev = torch.device("cuda:0")
+    torch.cuda.set_device(dev)
+    roof = project_record(lk, dev, wl, args.project, args.batch or 64, args.steps, args.warmup)
+    print(json.dumps({
+        "metric": "key/value producer (projection + rotary + append) us per call", "value": roof["us_per_launch"],
+        "unit": "us", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup, "ms_per_step": roof["us_per_launch"] / 1e3,
+        "higher_is_better": False, "dtype": "bf16", "data": "synthetic",
+        "config": {"workload": roof["workload"], "l2": "weight sets in rotation exceed L2"},
+        "roofline": roof}))
 
 
 def main():
@@ -572,6 +778,14 @@ def main():
                     help="P > 0: paged caches with P-row pages and a pool sized for the batch's lengths")
     ap.add_argument("--stream-sink", type=int, default=0,
                     help="s > 0: sink + recent-window caches with s sink tokens, cache size = context")
+    ap.add_argument("--shard", default="", choices=["", "batch", "heads"],
+                    help="split ONE seeded batch over the ranks by sequences or by kv heads (strong scaling); "
+                         "default: every rank runs its own replica of the workload (weak scaling)")
+    ap.add_argument("--extras", type=int, default=-1,
+                    help="1: also time the other workload shapes, prompt encoding and the key/value producer "
+                         "(default: only in the plain default run)")
+    ap.add_argument("--kernel-digests", action="store_true",
+                    help="print the source digests profiles/ncu_captures.json compares against, and exit")
     ap.add_argument("--ref-rows", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prefill", type=int, default=0,
@@ -580,6 +794,15 @@ def main():
                     help="D > 0: time the fused key/value producer for hidden width D instead")
     args = ap.parse_args()
     args.warmup = max(args.warmup, 3) if args.impl == "ours" else args.warmup
+    if args.kernel_digests:
+        for name, cap in load_captures().items():
+            if isinstance(cap, dict):
+                print(name, source_digest(cap["sources"]))
+        return
+    if args.extras < 0:   # the plain default run carries every workload shape
+        args.extras = int(args.workload == "llama7b" and not (args.batch or args.context or args.page_rows or
+                          args.stream_sink or args.shard or args.top_variant or args.kernel_kind or
+                          args.warmup_layers is not None or args.prefill or args.project))
     if args.impl == "reference":
         run_reference(args)
     else:

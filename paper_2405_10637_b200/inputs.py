@@ -115,3 +115,12 @@ def shard_batch(total_batch: int, rank: int, world: int):
     base, rem = divmod(total_batch, world)
     start = rank * base + min(rank, rem)
     return start, start + base + (1 if rank < rem else 0)
+
+
+def shard_heads(n_kv_heads: int, rank: int, world: int):
+    """Contiguous kv-head shard [start, stop) of this rank; a rank takes whole kv heads, hence whole
+    query groups (q heads [start * g, stop * g)), so no rank needs another's keys or values."""
+    if n_kv_heads % world:
+        raise ValueError(f"{n_kv_heads} kv heads do not split evenly over {world} ranks")
+    per = n_kv_heads // world
+    return rank * per, (rank + 1) * per

@@ -19,7 +19,7 @@ def bench():
 
 def args_for(**kw):
     base = dict(workload="llama7b", batch=0, context=0, warmup_layers=None, stream_sink=0, page_rows=0,
-                steps=10, warmup=3)
+                steps=10, warmup=3, shard="")
     base.update(kw)
     return argparse.Namespace(**base)
 
@@ -39,10 +39,47 @@ def test_workload_parameters(bench):
 def test_traffic_is_scaled_from_the_capture_only_where_it_applies(bench):
     alg = 17.9e9
     out = 512 * 32 * 128 * 2
-    t = bench.scaled_traffic("attn_alu_kernel", args_for(), alg, out)
+    caps = bench.load_captures()
+    t = bench.scaled_traffic("attn_alu_kernel", args_for(), alg, out, caps, check_sources=False)
     assert alg < t < 1.01 * alg                          # every K/V byte once, plus partials and write-backs
-    assert bench.scaled_traffic("attn_alu_kernel", args_for(page_rows=256), alg, out) is None
-    assert bench.scaled_traffic("attn_mma_kernel", args_for(workload="tinyllama"), 135.3e6, 524288) is not None
-    assert bench.scaled_traffic("attn_mma_kernel", args_for(workload="tinyllama", context=512), 67e6, 524288) is None
-    for cap in bench.NCU_CAPTURES.values():
-        assert os.path.exists(os.path.join(ROOT, cap["source"]))
+    f = lambda k, a, x, o: bench.scaled_traffic(k, a, x, o, caps, check_sources=False)
+    assert f("attn_alu_kernel", args_for(page_rows=256), alg, out) is None
+    assert f("attn_mma_kernel", args_for(workload="tinyllama"), 135.3e6, 524288) is not None
+    assert f("attn_mma_kernel", args_for(workload="tinyllama", context=512), 67e6, 524288) is None
+
+
+def test_captured_counters_are_the_ones_in_the_summaries(bench):
+    """bench.py takes the DRAM counters from profiles/ncu_captures.json; the figures there must be the
+    ones the ncu summaries beside it print (to the precision they print)."""
+    caps = bench.load_captures()
+    for name in ("attn_alu_kernel", "attn_mma_kernel"):
+        cap = caps[name]
+        text = open(os.path.join(ROOT, cap["source"])).read()
+        rows = {ln.split("|")[1].strip(): [c.strip() for c in ln.split("|")[2:-1]]
+                for ln in text.splitlines() if ln.startswith("| `dram__bytes")}
+        reads = [float(c.split()[0]) * 1e6 for c in rows["`dram__bytes_read.sum`"]]
+        writes = [float(c.split()[0]) * 1e6 for c in rows["`dram__bytes_write.sum`"]]
+        assert min(reads) - 0.02e6 <= cap["dram_read_bytes"] <= max(reads) + 0.02e6
+        assert min(writes) - 0.02e6 <= cap["dram_write_bytes"] <= max(writes) + 0.02e6
+        assert cap["output_bytes"] < cap["dram_write_bytes"] < 0.05 * cap["dram_read_bytes"]
+        assert 0.9 * cap["dram_read_bytes"] < cap["algorithmic_input_bytes"] <= cap["dram_read_bytes"]
+        for src in cap["sources"]:
+            assert os.path.exists(os.path.join(bench.CSRC, src))
+
+
+def test_a_capture_is_void_once_the_kernel_changed(bench):
+    caps = bench.load_captures()
+    caps = {k: dict(v) if isinstance(v, dict) else v for k, v in caps.items()}
+    caps["attn_alu_kernel"]["sources_digest"] = bench.source_digest(caps["attn_alu_kernel"]["sources"])
+    assert bench.scaled_traffic("attn_alu_kernel", args_for(), 17.9e9, 4e6, caps) is not None
+    caps["attn_alu_kernel"]["sources_digest"] = "0" * 16
+    assert bench.scaled_traffic("attn_alu_kernel", args_for(), 17.9e9, 4e6, caps) is None
+
+
+def test_largest_batch_that_fits(bench):
+    from paper_2405_10637_b200 import inputs as syn
+    wl = syn.WORKLOADS["llama30b"]
+    assert bench.largest_batch(wl, 4096, 2) == 825      # 109.05 MB per sequence and cache
+    assert bench.largest_batch(wl, 4096, 3) == 550
+    wl = syn.WORKLOADS["sweep7b"]
+    assert bench.largest_batch(wl, 8192, 32) == 41      # the standard transformer's 32 caches: 64 do not fit

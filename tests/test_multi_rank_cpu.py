@@ -1,5 +1,5 @@
-"""The N > 1 path on CPU (gloo, world size 2): batch sharding is exact and needs no data-path
-collective; timing aggregation is max over ranks, throughput is the sum of units over that time."""
+"""The N > 1 path on CPU (gloo, world size 2): sharding one batch by sequences or by kv heads is exact
+(the union of the ranks' results is the one-rank result, bit for bit) and needs no data-path collective; timing aggregation is max over ranks, throughput is the sum of units over that time."""
 import os
 import socket
 import subprocess
@@ -33,6 +33,47 @@ WORKER = textwrap.dedent("""
         covered = sorted(parts)
         assert covered[0][0] == 0 and covered[-1][1] == B
         assert all(a[1] == b[0] for a, b in zip(covered, covered[1:]))
+    # both shard rules, whole stack step: each rank steps ITS shard of one batch with the oracle; the
+    # union of the ranks' outputs, caches and lengths is what one rank computes for the whole batch
+    L, wm = 4, 2
+    qs = [syn.bits(syn.randn_bf16((B, Hq, d), 10 + l)) for l in range(L)]
+    plan = orc.plan(L, wm)
+    kn = [syn.bits(syn.randn_bf16((B, Hkv, d), 20 + l)) if plan["write_slot"][l] >= 0 else None for l in range(L)]
+    vn = [syn.bits(syn.randn_bf16((B, Hkv, d), 30 + l)) if plan["write_slot"][l] >= 0 else None for l in range(L)]
+    Ks = [syn.bits(syn.randn_bf16((B, Hkv, T, d), 40 + s)) for s in range(plan["n_slots"])]
+    Vs = [syn.bits(syn.randn_bf16((B, Hkv, T, d), 50 + s)) for s in range(plan["n_slots"])]
+    ln = np.array([0, 7, 38, 16, 1], np.int32)
+    cp = lambda xs: [None if x is None else np.ascontiguousarray(x) for x in xs]
+    fK, fV, fl = cp(Ks), cp(Vs), ln.copy()
+    full_out, _ = orc.stack_step(L, wm, qs, kn, vn, fK, fV, fl, 0.25)
+    g = Hq // Hkv
+    for rule in ("batch", "heads"):
+        if rule == "batch":
+            (b0, b1), (h0, h1) = syn.shard_batch(B, r, w), (0, Hkv)
+        else:
+            (b0, b1), (h0, h1) = (0, B), syn.shard_heads(Hkv, r, w)
+        cut = lambda x, hs: None if x is None else np.ascontiguousarray(x[b0:b1, hs[0]:hs[1]])
+        sK = [cut(x, (h0, h1)) for x in Ks]; sV = [cut(x, (h0, h1)) for x in Vs]
+        sl = ln[b0:b1].copy()
+        out, _ = orc.stack_step(L, wm, [cut(x, (h0 * g, h1 * g)) for x in qs], [cut(x, (h0, h1)) for x in kn],
+                                [cut(x, (h0, h1)) for x in vn], sK, sV, sl, 0.25)
+        got = [None] * w
+        dist.all_gather_object(got, (b0, b1, h0, h1, out, sK, sV, sl))
+        if r == 0:
+            uo = [np.full_like(x, np.nan) for x in full_out]
+            uK = [np.zeros_like(x) for x in fK]; uV = [np.zeros_like(x) for x in fV]
+            ul = np.full(B, -1, np.int32)
+            for (a0, a1, c0, c1, o, pk, pv, pl) in got:
+                for l in range(L):
+                    uo[l][a0:a1, c0 * g:c1 * g] = o[l]
+                for s in range(len(fK)):
+                    uK[s][a0:a1, c0:c1] = pk[s]; uV[s][a0:a1, c0:c1] = pv[s]
+                ul[a0:a1] = pl
+            for l in range(L):
+                assert np.array_equal(uo[l], full_out[l]), (rule, l)
+            for s in range(len(fK)):
+                assert np.array_equal(uK[s], fK[s]) and np.array_equal(uV[s], fV[s]), (rule, s)
+            assert np.array_equal(ul, fl), rule
     ms = 10.0 + 5.0 * r                               # rank 1 is the slow one
     assert multi.max_over_ranks(ms) == 15.0
     thr = multi.job_throughput(float(hi - lo), ms)
@@ -51,6 +92,17 @@ def test_shard_batch_partitions_exactly():
             assert all(a[1] == b[0] for a, b in zip(parts, parts[1:]))
             sizes = [b - a for a, b in parts]
             assert max(sizes) - min(sizes) <= 1
+
+
+def test_shard_heads_takes_whole_query_groups():
+    for Hkv, w in ((4, 1), (4, 2), (4, 4), (32, 8), (52, 4)):
+        parts = [syn.shard_heads(Hkv, r, w) for r in range(w)]
+        assert parts[0][0] == 0 and parts[-1][1] == Hkv
+        assert all(a[1] == b[0] for a, b in zip(parts, parts[1:]))
+        assert len({b - a for a, b in parts}) == 1
+    import pytest
+    with pytest.raises(ValueError):
+        syn.shard_heads(52, 0, 8)
 
 
 def test_two_ranks_gloo():
