@@ -394,13 +394,17 @@ int lckv_decode_attention_static(const void* k, const void* v, const int32_t* le
  * not show.  kind 0: independent 16-byte loads from every thread; kind 2: 32-byte loads
  * (src 32-byte aligned) marked evict-first; kind 1: 8 KB bulk copies into
  * per-warp shared-memory rings, the way the attention kernels stream K and V (bytes beyond the last
- * whole 8 KB are not read).  *dev_sum (device uint32, not cleared) receives a checksum so that the
+ * whole 8 KB are not read).  `repeats` >= 1 passes over the buffer are made in one launch: with a buffer
+ * smaller than the L2 the passes after the first measure the L2's read bandwidth, the ceiling of a layer
+ * that re-reads a cache the previous layer left there.  l2_keep in [0, 1] (kind 1 only) is the fraction of
+ * lines the copies mark evict-last, as the attention kernels do for a cache that several layers read; the
+ * rest is marked evict-first.  *dev_sum (device uint32, not cleared) receives a checksum so that the
  * reads cannot be optimised away: kinds 0 and 2 add the wrapped sum of all 32-bit words, kind 1 the first
- * word of every piece.  *dev_status (device int32) is set to LCKV_ETIMEOUT if a bounded wait of kind 1
+ * word of every piece (each once per pass).  *dev_status (device int32) is set to LCKV_ETIMEOUT if a bounded wait of kind 1
  * runs out.  Time it with events on `stream`.  Errors: EINVAL, ECUDA.
  */
-int lckv_read_stream_probe(const void* src, size_t bytes, int32_t kind, uint32_t* dev_sum,
-                           int32_t* dev_status, void* stream);
+int lckv_read_stream_probe(const void* src, size_t bytes, int32_t kind, int32_t repeats, float l2_keep,
+                           uint32_t* dev_sum, int32_t* dev_status, void* stream);
 
 /* Short English name of a status code. */
 const char* lckv_status_string(int status);

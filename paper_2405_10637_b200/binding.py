@@ -56,7 +56,7 @@ SIGNATURES = {
     "lckv_prefill_iteration": (C.c_int, [_vp, _vpp, _vpp, _vpp, _vpp, _i32, _i32, _vp]),
     "lckv_decode_attention_static": (C.c_int, [_vp, _vp, _vp, _vp, _vp, _vp, _vp, _i32, _i32, _i32,
                                               _i32, C.c_int64, _i32, C.c_float, _i32, _vp]),
-    "lckv_read_stream_probe": (C.c_int, [_vp, C.c_size_t, _i32, _vp, _vp, _vp]),
+    "lckv_read_stream_probe": (C.c_int, [_vp, C.c_size_t, _i32, _i32, C.c_float, _vp, _vp, _vp]),
     "lckv_status_string": (C.c_char_p, [C.c_int]),
     "lckv_last_cuda_error": (C.c_int, []),
 }
@@ -147,11 +147,11 @@ def lckv_decode_attention_static(k, v, lens, q, out, mode, lse=None, dev_status=
     return out
 
 
-def lckv_read_stream_probe(src, nbytes, kind, dev_sum, dev_status, stream=None):
-    """Read-only stream over the first nbytes of the CUDA tensor `src`; dev_sum (uint32/int32 [1]) and
-    dev_status (int32 [1]) are CUDA tensors."""
-    _chk(lib().lckv_read_stream_probe(_ptr(src), nbytes, kind, _ptr(dev_sum), _ptr(dev_status),
-                                      _stream(stream)), "lckv_read_stream_probe")
+def lckv_read_stream_probe(src, nbytes, kind, dev_sum, dev_status, repeats=1, l2_keep=0.0, stream=None):
+    """Read-only stream over the first nbytes of the CUDA tensor `src`, `repeats` passes in one launch;
+    dev_sum (uint32/int32 [1]) and dev_status (int32 [1]) are CUDA tensors."""
+    _chk(lib().lckv_read_stream_probe(_ptr(src), nbytes, kind, repeats, l2_keep, _ptr(dev_sum),
+                                      _ptr(dev_status), _stream(stream)), "lckv_read_stream_probe")
 
 
 class Cache:

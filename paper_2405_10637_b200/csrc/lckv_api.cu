@@ -1243,10 +1243,11 @@ int lckv_prefill_iteration(lckv_cache_t* c, const void* const* q_layers, void* c
     return LCKV_OK;
 }
 
-int lckv_read_stream_probe(const void* src, size_t bytes, int32_t kind, uint32_t* dev_sum,
-                           int32_t* dev_status, void* stream)
+int lckv_read_stream_probe(const void* src, size_t bytes, int32_t kind, int32_t repeats, float l2_keep,
+                           uint32_t* dev_sum, int32_t* dev_status, void* stream)
 {
-    if (!src || !dev_sum || !dev_status || bytes < 16) return LCKV_EINVAL;
+    if (!src || !dev_sum || !dev_status || bytes < 16 || repeats < 1) return LCKV_EINVAL;
+    if (!(l2_keep >= 0.f && l2_keep <= 1.f)) return LCKV_EINVAL;
     if (((uintptr_t)src & 15) || ((uintptr_t)dev_sum & 3) || ((uintptr_t)dev_status & 3)) return LCKV_EINVAL;
     if (kind < 0 || kind > 2 || (kind == 2 && ((uintptr_t)src & 31))) return LCKV_EINVAL;
     int sm = 0;
@@ -1255,10 +1256,10 @@ int lckv_read_stream_probe(const void* src, size_t bytes, int32_t kind, uint32_t
     if (kind == 0) {
         // 8 resident blocks of 256 threads per SM: 16 KB of loads in flight per SM and loop trip
         lckv::read_stream_ldg_kernel<<<sm * 8, lckv::kProbeThreads, 0, st>>>(
-            static_cast<const uint4*>(src), (uint64_t)(bytes / 16), dev_sum);
+            static_cast<const uint4*>(src), (uint64_t)(bytes / 16), dev_sum, repeats);
     } else if (kind == 2) {
         lckv::read_stream_ldg32_kernel<<<sm * 8, lckv::kProbeThreads, 0, st>>>(
-            static_cast<const uint8_t*>(src), (uint64_t)(bytes / 32), dev_sum);
+            static_cast<const uint8_t*>(src), (uint64_t)(bytes / 32), dev_sum, repeats);
     } else {
         static std::once_flag once[64];
         int dev = 0;
@@ -1271,7 +1272,8 @@ int lckv_read_stream_probe(const void* src, size_t bytes, int32_t kind, uint32_t
         });
         if (!ok) return LCKV_ECUDA;
         lckv::read_stream_bulk_kernel<<<sm, lckv::kProbeThreads, lckv::kProbeSmemBytes, st>>>(
-            static_cast<const uint8_t*>(src), (uint64_t)(bytes / lckv::kProbePiece), dev_sum, dev_status);
+            static_cast<const uint8_t*>(src), (uint64_t)(bytes / lckv::kProbePiece), dev_sum, dev_status, repeats,
+            l2_keep);
     }
     return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
 }

@@ -13,7 +13,9 @@
 //  * A pair that falls entirely inside one worker's range is normalised and written directly.
 //    A pair cut by a range boundary leaves an fp32 partial (m, l, o) per contributing worker; the
 //    contributor that arrives last (atomic ticket, no waiting) merges them with the log-sum-exp
-//    rule in a fixed order and writes the row.
+//    rule in a fixed order and writes the row.  A worker posts its ticket when its part is done
+//    but looks at the answer only after its last tile, so the round trip of the atomic and the merge
+//    itself never sit between two tiles of its range.
 #pragma once
 #include "lckv_device.cuh"
 
@@ -71,11 +73,13 @@ struct TileCursor {
     int32_t b, h;
     uint32_t t, nt;   // tile within the pair; tiles per pair of sequence b
     int32_t nv;       // visible rows of sequence b
+    uint32_t pre0;    // tiles (per pair index) of the sequences before b
 };
 
 __device__ __forceinline__ void cursor_load(TileCursor& c, const AttnParams& p)
 {
-    c.nt = __ldg(p.pre + c.b + 1) - __ldg(p.pre + c.b);
+    c.pre0 = __ldg(p.pre + c.b);
+    c.nt = __ldg(p.pre + c.b + 1) - c.pre0;
     c.nv = visible_rows(__ldg(p.lens + c.b), p.mode, p.T_cap);
 }
 
@@ -148,13 +152,13 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
     const bool has_work = (uint64_t)w < n_eff;
     uint64_t lo = 0, hi = 0;
     TileCursor cc;
-    cc.b = 0; cc.h = 0; cc.t = 0; cc.nt = 0; cc.nv = 0;
+    cc.b = 0; cc.h = 0; cc.t = 0; cc.nt = 0; cc.nv = 0; cc.pre0 = 0;
     if (has_work) {
         lo = (uint64_t)w * total / n_eff;
         hi = (uint64_t)(w + 1) * total / n_eff;
         cc.b = __ldg(p.start_b + w);
         cursor_load(cc, p);
-        const uint64_t rel = lo - (uint64_t)__ldg(p.pre + cc.b) * (uint64_t)H;
+        const uint64_t rel = lo - (uint64_t)cc.pre0 * (uint64_t)H;
         cc.h = (int32_t)(rel / cc.nt);
         cc.t = (uint32_t)(rel % cc.nt);
     }
@@ -216,9 +220,7 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
 #pragma unroll
     for (int j = 0; j < 4; ++j) o2[j] = 0ull;
 #endif
-    auto load_q = [&](const TileCursor& c) {
-        const uint4 raw =
-            __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)c.b * H + c.h) * D) + a);
+    auto set_q = [&](const uint4 raw) {
         qf[0] = bf16lo(raw.x) * p.scale_log2; qf[1] = bf16hi(raw.x) * p.scale_log2;
         qf[2] = bf16lo(raw.y) * p.scale_log2; qf[3] = bf16hi(raw.y) * p.scale_log2;
         qf[4] = bf16lo(raw.z) * p.scale_log2; qf[5] = bf16hi(raw.z) * p.scale_log2;
@@ -228,15 +230,110 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
         for (int j = 0; j < 4; ++j) q2[j] = pack_f32x2(qf[2 * j], qf[2 * j + 1]);
 #endif
     };
-    load_q(cc);
+    set_q(__ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)cc.b * H + cc.h) * D) + a));
     uint32_t seg_t0 = cc.t;
     float m_run = -INFINITY, l_run = 0.f;
     float o[8];
 #pragma unroll
     for (int k = 0; k < 8; ++k) o[k] = 0.f;
 
+    // Tickets posted for the (at most two) pairs this worker shares with others: the pair its range
+    // starts in the middle of (record 0) and the pair it ends in the middle of (record 1).
+    struct Pending { int32_t ticket, n, first_odd, b, h; uint32_t c_first; bool armed; };
+    Pending pend0 = {0, 0, 0, 0, 0, 0u, false}, pend1 = pend0;
+    // Which workers share a pair: worked out when the worker enters a pair that its range cuts (at
+    // most its first and its last), so that the divisions are off the path that ends the kernel.
+    struct Split { uint32_t c_first; int32_t n_parts, first_odd; };
+    auto split_of = [&](const TileCursor& c) {
+        const uint64_t gs = (uint64_t)c.pre0 * (uint64_t)H + (uint64_t)c.h * c.nt;  // the pair's first global tile
+        const uint64_t ge = gs + c.nt;
+        Split sp;
+        sp.c_first = (uint32_t)(((gs + 1) * n_eff - 1) / total);
+        const uint32_t c_last = (uint32_t)((ge * n_eff - 1) / total);
+        const uint64_t lo_first = (uint64_t)sp.c_first * total / n_eff;
+        sp.first_odd = (gs != lo_first) ? 1 : 0;  // which record of c_first belongs to this pair
+        sp.n_parts = (int32_t)(c_last - sp.c_first) + 1;
+        return sp;
+    };
+    Split cur = {0u, 1, 0}, nxt = cur;
+    if (cc.t != 0 || n_tiles < cc.nt) cur = split_of(cc);   // the first pair is cut by this range
+    bool first_seg = true;                                  // still in the segment that starts at lo
+    float l_tot = 0.f, m_fin = 0.f;   // with o[]: the (unnormalised) result being stored or merged
+
+    // o / l_tot, lse from (m_fin, l_tot) -> output row of pair (b, h)
+    auto write_row = [&](int b, int h) {
+        const float inv = 1.0f / l_tot;
+        const size_t row = (size_t)b * H + h;
+        if (lane < LPR) {
+            if (p.out_f32) {
+                float4* dst = reinterpret_cast<float4*>(static_cast<float*>(p.out) + row * D);
+                dst[2 * lane] = make_float4(o[0] * inv, o[1] * inv, o[2] * inv, o[3] * inv);
+                dst[2 * lane + 1] = make_float4(o[4] * inv, o[5] * inv, o[6] * inv, o[7] * inv);
+            } else {
+                uint4 pk;
+                pk.x = pack_bf16x2(o[0] * inv, o[1] * inv);
+                pk.y = pack_bf16x2(o[2] * inv, o[3] * inv);
+                pk.z = pack_bf16x2(o[4] * inv, o[5] * inv);
+                pk.w = pack_bf16x2(o[6] * inv, o[7] * inv);
+                reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + row * D)[lane] = pk;
+            }
+        }
+        if (p.lse && lane == 0) p.lse[row] = (m_fin + lg2(l_tot)) * 0.6931471805599453f;
+    };
+    // (o, m_fin, l_tot) -> a partial record
+    auto store_record = [&](float* rec) {
+        if (lane < LPR) {
+            reinterpret_cast<float4*>(rec)[2 * lane] = make_float4(o[0], o[1], o[2], o[3]);
+            reinterpret_cast<float4*>(rec)[2 * lane + 1] = make_float4(o[4], o[5], o[6], o[7]);
+        }
+        if (lane == 0) { rec[D] = m_fin; rec[D + 1] = l_tot; }
+    };
+    // Merge of n records in a fixed order, in one pass with a running maximum: record i is the one of
+    // worker first_w + i * step (its second record if i == 0 and first_slot is set).  Record
+    // addresses do not depend on loaded data, so the unrolled loop keeps several L2 round trips in
+    // flight.  Leaves the merged (unnormalised) values in o, l_tot, m_fin.
+    auto merge_records = [&](int n, uint32_t first_w, int step, int first_slot) {
+        const float* rec0 = p.partials + (size_t)(2 * first_w) * REC;
+        const size_t rstride = (size_t)(2 * step) * REC;
+        float M = -INFINITY, Lsum = 0.f, acc[8];
+#pragma unroll
+        for (int k = 0; k < 8; ++k) acc[k] = 0.f;
+#pragma unroll 4
+        for (int i = 0; i < n; ++i) {
+            const float* r = rec0 + (size_t)i * rstride + (i == 0 ? (size_t)first_slot * REC : 0);
+            const float2 ml = __ldcg(reinterpret_cast<const float2*>(r + D));
+            float4 x0 = make_float4(0.f, 0.f, 0.f, 0.f), x1 = x0;
+            if (lane < LPR) {
+                x0 = __ldcg(reinterpret_cast<const float4*>(r) + 2 * lane);
+                x1 = __ldcg(reinterpret_cast<const float4*>(r) + 2 * lane + 1);
+            }
+            const float Mn = fmaxf(M, ml.x);
+            const float ca = ex2(M - Mn), cb = ex2(ml.x - Mn);   // ex2(-inf) = 0 for the first record
+            M = Mn;
+            Lsum = fmaf(Lsum, ca, ml.y * cb);
+            acc[0] = fmaf(acc[0], ca, x0.x * cb); acc[1] = fmaf(acc[1], ca, x0.y * cb);
+            acc[2] = fmaf(acc[2], ca, x0.z * cb); acc[3] = fmaf(acc[3], ca, x0.w * cb);
+            acc[4] = fmaf(acc[4], ca, x1.x * cb); acc[5] = fmaf(acc[5], ca, x1.y * cb);
+            acc[6] = fmaf(acc[6], ca, x1.z * cb); acc[7] = fmaf(acc[7], ca, x1.w * cb);
+        }
+#pragma unroll
+        for (int k = 0; k < 8; ++k) o[k] = acc[k];
+        l_tot = Lsum;
+        m_fin = M;
+    };
+
     for (uint32_t tile = 0; tile < n_tiles; ++tile) {
         const int rows = min(R, cc.nv - (int)cc.t * R);
+        const bool pair_end = (cc.t + 1 == cc.nt);
+        const bool last = (tile + 1 == n_tiles);
+        // the next pair's query is fetched while this pair's last tile is worked on
+        TileCursor cn = cc;
+        uint4 q_next = make_uint4(0, 0, 0, 0);
+        if (pair_end && !last) {
+            cursor_next(cn, p, H);
+            if (n_tiles - (tile + 1) < cn.nt) nxt = split_of(cn);   // the range ends inside the next pair
+            q_next = __ldg(reinterpret_cast<const uint4*>(p.q + ((size_t)cn.b * H + cn.h) * D) + a);
+        }
 
         // ---- K tile: scores -----------------------------------------------------------------
         if (!mbar_wait_bounded(bars + 8 * cslot, cphase, p.wait_limit)) { ok = false; break; }
@@ -375,8 +472,6 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
         if (cslot == 0) cphase ^= 1;
 
         // ---- end of this worker's part of the pair? -----------------------------------------
-        const bool pair_end = (cc.t + 1 == cc.nt);
-        const bool last = (tile + 1 == n_tiles);
         if (pair_end || last) {
             // everything this worker saw of the pair: reduce over row groups and lanes
 #if LCKV_ALU_FFMA2
@@ -387,126 +482,69 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
             for (int off = LPR; off < 32; off <<= 1)
 #pragma unroll
                 for (int k = 0; k < 8; ++k) o[k] += __shfl_xor_sync(FULL, o[k], off);
-            float l_tot = l_run;
+            l_tot = l_run;
 #pragma unroll
             for (int off = 16; off >= 1; off >>= 1) l_tot += __shfl_xor_sync(FULL, l_tot, off);
             l_tot *= (1.0f / DUP);
-            float m_fin = m_run;
+            m_fin = m_run;
 
             const bool complete = pair_end && seg_t0 == 0;
-            bool write_row = complete;
-            if (!complete) {
-                const uint64_t gs = (uint64_t)__ldg(p.pre + cc.b) * (uint64_t)H +
-                                    (uint64_t)cc.h * cc.nt;  // the pair's first global tile
-                const uint64_t ge = gs + cc.nt;
-                const uint32_t c_first = (uint32_t)(((gs + 1) * n_eff - 1) / total);
-                const uint32_t c_last = (uint32_t)((ge * n_eff - 1) / total);
-                const bool at_lo = (gs + seg_t0 == lo);
-                float* rec = p.partials + (size_t)(2 * w + (at_lo ? 0 : 1)) * REC;
-                if (lane < LPR) {
-                    reinterpret_cast<float4*>(rec)[2 * lane] = make_float4(o[0], o[1], o[2], o[3]);
-                    reinterpret_cast<float4*>(rec)[2 * lane + 1] =
-                        make_float4(o[4], o[5], o[6], o[7]);
-                }
-                if (lane == 0) { rec[D] = m_fin; rec[D + 1] = l_tot; }
-                __threadfence();
-                __syncwarp();
-                // Merge of n records in a fixed order: record i is the one of worker
-                // first_w + i * step (its second record if i == 0 and first_slot is set).  Record
-                // addresses do not depend on loaded data, so the unrolled loops keep several L2 round
-                // trips in flight.  Leaves the merged (unnormalised) values in o, l_tot, m_fin.
-                auto merge_records = [&](int n, uint32_t first_w, int step, int first_slot) {
-                    const float* rec0 = p.partials + (size_t)(2 * first_w) * REC;
-                    const size_t rstride = (size_t)(2 * step) * REC;
-                    float M = -INFINITY;
-#pragma unroll 4
-                    for (int i = 0; i < n; ++i) {
-                        const float* r = rec0 + (size_t)i * rstride + (i == 0 ? (size_t)first_slot * REC : 0);
-                        M = fmaxf(M, __ldcg(r + D));
-                    }
-                    float Lsum = 0.f, acc[8];
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) acc[k] = 0.f;
-#pragma unroll 4
-                    for (int i = 0; i < n; ++i) {
-                        const float* r = rec0 + (size_t)i * rstride + (i == 0 ? (size_t)first_slot * REC : 0);
-                        const float2 ml = __ldcg(reinterpret_cast<const float2*>(r + D));
-                        const float wgt = ex2(ml.x - M);
-                        Lsum = fmaf(ml.y, wgt, Lsum);
-                        if (lane < LPR) {
-                            const float4 x0 = __ldcg(reinterpret_cast<const float4*>(r) + 2 * lane);
-                            const float4 x1 =
-                                __ldcg(reinterpret_cast<const float4*>(r) + 2 * lane + 1);
-                            acc[0] = fmaf(x0.x, wgt, acc[0]); acc[1] = fmaf(x0.y, wgt, acc[1]);
-                            acc[2] = fmaf(x0.z, wgt, acc[2]); acc[3] = fmaf(x0.w, wgt, acc[3]);
-                            acc[4] = fmaf(x1.x, wgt, acc[4]); acc[5] = fmaf(x1.y, wgt, acc[5]);
-                            acc[6] = fmaf(x1.z, wgt, acc[6]); acc[7] = fmaf(x1.w, wgt, acc[7]);
-                        }
-                    }
-#pragma unroll
-                    for (int k = 0; k < 8; ++k) o[k] = acc[k];
-                    l_tot = Lsum;
-                    m_fin = M;
-                };
-                const uint64_t lo_first = (uint64_t)c_first * total / n_eff;
-                const int first_odd = (gs != lo_first) ? 1 : 0;  // which record of c_first belongs to this pair
-                const int n_parts = (int)(c_last - c_first) + 1;
+            if (complete) {
+                write_row(cc.b, cc.h);
+            } else {
+                const uint32_t c_first = cur.c_first;
+                const int first_odd = cur.first_odd, n_parts = cur.n_parts;
+                const bool at_lo = first_seg;
+                store_record(p.partials + (size_t)(2 * w + (at_lo ? 0 : 1)) * REC);
                 // Few parts: the contributor that arrives last merges them all.  Many parts (few
                 // pairs, long sequences): two levels - the contributors of a pair form chunks of
                 // kAluChunk consecutive workers; the last arriver of a chunk merges the chunk's records
                 // into the record of the chunk's first worker, and the last chunk to finish merges
                 // the chunk records.  Same fixed order either way.
                 const bool two_level = n_parts > kAluTreeMin && p.counters2 != nullptr;
-                const int kk = (int)((uint32_t)w - c_first);         // this contributor's index in the pair
-                const int ck = (kk / kAluChunk) * kAluChunk;         // its chunk's first index
-                const uint32_t cw = c_first + (uint32_t)ck;          // chunk's first worker
-                const int first_rec = (ck == 0) ? first_odd : 0;
-                int32_t* tk = two_level ? p.counters2 + 2 * cw + first_rec : p.counters + c_first;
-                int n = two_level ? min(kAluChunk, n_parts - ck) : n_parts;
-                uint32_t fw = two_level ? cw : c_first;
-                int step = 1, fslot = two_level ? first_rec : first_odd;
-                for (int round = two_level ? 0 : 1; round < 2; ++round) {
-                    int ticket = 0;
-                    if (lane == 0) ticket = atomicAdd(tk, 1);
-                    ticket = __shfl_sync(FULL, ticket, 0);
-                    if (ticket != n - 1) break;          // someone else arrives later and merges
-                    __threadfence();
-                    merge_records(n, fw, step, fslot);
-                    if (lane == 0) *tk = 0;              // ready for the next launch
-                    if (round == 1) { write_row = true; break; }
-                    // the chunk's result becomes the record of the chunk's first worker
-                    float* crec = p.partials + (size_t)(2 * cw + first_rec) * REC;
-                    if (lane < LPR) {
-                        reinterpret_cast<float4*>(crec)[2 * lane] = make_float4(o[0], o[1], o[2], o[3]);
-                        reinterpret_cast<float4*>(crec)[2 * lane + 1] = make_float4(o[4], o[5], o[6], o[7]);
+                if (!two_level) {
+                    // Post the ticket now (the release and the atomic's flight overlap with the copies
+                    // of the next tiles, already on their way); the answer is looked at after the last
+                    // tile.  Each ticket goes straight into its own variable: nothing may consume the
+                    // atomic's result here, or the warp would wait for the round trip after all.
+                    __syncwarp();   // the record's stores (all lanes) are ordered before lane 0's release
+                    if (at_lo) {
+                        if (lane == 0) pend0.ticket = atom_add_acq_rel_gpu(p.counters + c_first, 1);
+                        pend0.n = n_parts; pend0.first_odd = first_odd; pend0.b = cc.b; pend0.h = cc.h;
+                        pend0.c_first = c_first; pend0.armed = true;
+                    } else {
+                        if (lane == 0) pend1.ticket = atom_add_acq_rel_gpu(p.counters + c_first, 1);
+                        pend1.n = n_parts; pend1.first_odd = first_odd; pend1.b = cc.b; pend1.h = cc.h;
+                        pend1.c_first = c_first; pend1.armed = true;
                     }
-                    if (lane == 0) { crec[D] = m_fin; crec[D + 1] = l_tot; }
+                } else {
                     __threadfence();
                     __syncwarp();
-                    tk = p.counters + c_first; n = (n_parts + kAluChunk - 1) / kAluChunk; fw = c_first;
-                    step = kAluChunk; fslot = first_odd;
-                }
-            }
-            if (write_row) {
-                const float inv = 1.0f / l_tot;
-                const size_t row = (size_t)cc.b * H + cc.h;
-                if (lane < LPR) {
-                    if (p.out_f32) {
-                        float4* dst =
-                            reinterpret_cast<float4*>(static_cast<float*>(p.out) + row * D);
-                        dst[2 * lane] = make_float4(o[0] * inv, o[1] * inv, o[2] * inv, o[3] * inv);
-                        dst[2 * lane + 1] =
-                            make_float4(o[4] * inv, o[5] * inv, o[6] * inv, o[7] * inv);
-                    } else {
-                        uint4 pk;
-                        pk.x = pack_bf16x2(o[0] * inv, o[1] * inv);
-                        pk.y = pack_bf16x2(o[2] * inv, o[3] * inv);
-                        pk.z = pack_bf16x2(o[4] * inv, o[5] * inv);
-                        pk.w = pack_bf16x2(o[6] * inv, o[7] * inv);
-                        reinterpret_cast<uint4*>(static_cast<uint16_t*>(p.out) + row * D)[lane] = pk;
+                    const int kk = (int)((uint32_t)w - c_first);         // this contributor's index in the pair
+                    const int ck = (kk / kAluChunk) * kAluChunk;         // its chunk's first index
+                    const uint32_t cw = c_first + (uint32_t)ck;          // chunk's first worker
+                    const int first_rec = (ck == 0) ? first_odd : 0;
+                    int32_t* tk = p.counters2 + 2 * cw + first_rec;
+                    int n = min(kAluChunk, n_parts - ck);
+                    uint32_t fw = cw;
+                    int step = 1, fslot = first_rec;
+                    for (int round = 0; round < 2; ++round) {
+                        int ticket = 0;
+                        if (lane == 0) ticket = atomicAdd(tk, 1);
+                        ticket = __shfl_sync(FULL, ticket, 0);
+                        if (ticket != n - 1) break;          // someone else arrives later and merges
+                        __threadfence();
+                        merge_records(n, fw, step, fslot);
+                        if (lane == 0) *tk = 0;              // ready for the next launch
+                        if (round == 1) { write_row(cc.b, cc.h); break; }
+                        // the chunk's result becomes the record of the chunk's first worker
+                        store_record(p.partials + (size_t)(2 * cw + first_rec) * REC);
+                        __threadfence();
+                        __syncwarp();
+                        tk = p.counters + c_first; n = (n_parts + kAluChunk - 1) / kAluChunk; fw = c_first;
+                        step = kAluChunk; fslot = first_odd;
                     }
                 }
-                if (p.lse && lane == 0) p.lse[row] = (m_fin + lg2(l_tot)) * 0.6931471805599453f;
             }
             m_run = -INFINITY;
             l_run = 0.f;
@@ -518,8 +556,23 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
 #endif
         }
         if (!last) {
-            cursor_next(cc, p, H);
-            if (pair_end) { load_q(cc); seg_t0 = 0; }
+            cc = pair_end ? cn : cc;
+            if (pair_end) { set_q(q_next); seg_t0 = 0; cur = nxt; first_seg = false; }
+            else cursor_next(cc, p, H);
+        }
+    }
+
+    // The tickets posted above: whoever finds itself the last contributor of a pair merges it.
+    if (ok) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const Pending& pd = i == 0 ? pend0 : pend1;
+            if (!pd.armed) continue;
+            const int ticket = __shfl_sync(FULL, pd.ticket, 0);
+            if (ticket != pd.n - 1) continue;            // someone else arrives later and merges
+            merge_records(pd.n, pd.c_first, 1, pd.first_odd);
+            if (lane == 0) p.counters[pd.c_first] = 0;   // ready for the next launch
+            write_row(pd.b, pd.h);
         }
     }
 

@@ -84,13 +84,15 @@ struct RowCursor {
     int32_t b, h;      // sequence; pair within the sequence
     uint32_t t, nt;    // tile within the pair; tiles per pair of sequence b
     int32_t nv;        // visible rows of sequence b
+    uint32_t pre0;     // tiles (per pair index) of the sequences before b
     int32_t kvh, sub;  // kv head the pair reads; index of the pair among the pairs of that kv head
     int64_t row;       // cache row (of the [B*H_kv*T_cap, D] view) where the tile starts
 };
 
 __device__ __forceinline__ void rcursor_load(RowCursor& c, const AttnParams& p)
 {
-    c.nt = __ldg(p.pre + c.b + 1) - __ldg(p.pre + c.b);
+    c.pre0 = __ldg(p.pre + c.b);
+    c.nt = __ldg(p.pre + c.b + 1) - c.pre0;
     c.nv = visible_rows(__ldg(p.lens + c.b), p.mode, p.T_cap);
 }
 
@@ -167,13 +169,13 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
     const bool has_work = (uint64_t)w < n_eff;
     uint64_t lo = 0, hi = 0;
     RowCursor cc;
-    cc.b = 0; cc.h = 0; cc.t = 0; cc.nt = 0; cc.nv = 0; cc.kvh = 0; cc.sub = 0; cc.row = 0;
+    cc.b = 0; cc.h = 0; cc.t = 0; cc.nt = 0; cc.nv = 0; cc.pre0 = 0; cc.kvh = 0; cc.sub = 0; cc.row = 0;
     if (has_work) {
         lo = (uint64_t)w * total / n_eff;
         hi = (uint64_t)(w + 1) * total / n_eff;
         cc.b = __ldg(p.start_b + w);
         rcursor_load(cc, p);
-        const uint64_t rel = lo - (uint64_t)__ldg(p.pre + cc.b) * (uint64_t)H;
+        const uint64_t rel = lo - (uint64_t)cc.pre0 * (uint64_t)H;
         cc.h = (int32_t)(rel / cc.nt);
         cc.t = (uint32_t)(rel % cc.nt);
         rcursor_seek(cc, p, mp.groups_per_kv, R);
@@ -227,17 +229,17 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
     bool ok = true;
 
     // Q^T fragments of the pair's 8 query heads: lane holds query g4, dims 2*c4 (+1) (+8) per k-step.
-    uint32_t qb[KS][2];
-    auto load_q = [&](const RowCursor& c) {
+    uint32_t qb[KS][2], qn[KS][2];
+    auto load_q = [&](const RowCursor& c, uint32_t (&dst)[KS][2]) {
         const uint16_t* qp = p.q + ((size_t)c.b * mp.n_q_heads + (size_t)c.h * HP + g4) * D + 2 * c4;
         const bool real = g4 < HP;
 #pragma unroll
         for (int ks = 0; ks < KS; ++ks) {
-            qb[ks][0] = real ? __ldg(reinterpret_cast<const uint32_t*>(qp + ks * 16)) : 0u;
-            qb[ks][1] = real ? __ldg(reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8)) : 0u;
+            dst[ks][0] = real ? __ldg(reinterpret_cast<const uint32_t*>(qp + ks * 16)) : 0u;
+            dst[ks][1] = real ? __ldg(reinterpret_cast<const uint32_t*>(qp + ks * 16 + 8)) : 0u;
         }
     };
-    load_q(cc);
+    load_q(cc, qb);
     uint32_t seg_t0 = cc.t;
     // running state for this lane's two queries (2*c4, 2*c4+1)
     float m_run[2] = {-INFINITY, -INFINITY}, l_run[2] = {0.f, 0.f};
@@ -247,8 +249,132 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
 #pragma unroll
         for (int i = 0; i < 4; ++i) o[mt][i] = 0.f;
 
+    // Tickets posted for the (at most two) pairs this worker shares with others: the pair its range
+    // starts in the middle of (record 0) and the pair it ends in the middle of (record 1).  A ticket is
+    // posted when the worker's part is done and looked at only after its last tile.
+    struct Pending { int32_t ticket, n, first_odd, b, h; uint32_t c_first; bool armed; };
+    Pending pend0 = {0, 0, 0, 0, 0, 0u, false}, pend1 = pend0;
+    // Which workers share a pair: worked out when the worker enters a pair that its range cuts (at
+    // most its first and its last), so that the divisions are off the path that ends the kernel.
+    struct Split { uint32_t c_first; int32_t n_parts, first_odd; };
+    auto split_of = [&](const RowCursor& c) {
+        const uint64_t gs = (uint64_t)c.pre0 * (uint64_t)H + (uint64_t)c.h * c.nt;  // the pair's first global tile
+        const uint64_t ge = gs + c.nt;
+        Split sp;
+        sp.c_first = (uint32_t)(((gs + 1) * n_eff - 1) / total);
+        const uint32_t c_last = (uint32_t)((ge * n_eff - 1) / total);
+        const uint64_t lo_first = (uint64_t)sp.c_first * total / n_eff;
+        sp.first_odd = (gs != lo_first) ? 1 : 0;  // which record of c_first belongs to this pair
+        sp.n_parts = (int32_t)(c_last - sp.c_first) + 1;
+        return sp;
+    };
+    Split cur = {0u, 1, 0}, nxt = cur;
+    if (cc.t != 0 || n_tiles < cc.nt) cur = split_of(cc);   // the first pair is cut by this range
+    bool first_seg = true;                                  // still in the segment that starts at lo
+    float l_tot[2] = {0.f, 0.f}, m_fin[2] = {0.f, 0.f};   // with o[][]: the result being stored or merged
+
+    // o / l_tot, lse from (m_fin, l_tot) -> the output rows of pair (b, h)
+    auto write_rows = [&](int b, int h) {
+        const float inv0 = 1.0f / l_tot[0], inv1 = 1.0f / l_tot[1];
+        const size_t row0 = (size_t)b * mp.n_q_heads + (size_t)h * HP;  // first q head
+        const bool col0 = 2 * c4 < HP, col1 = 2 * c4 + 1 < HP;
+        if (p.out_f32) {
+            float* ob = static_cast<float*>(p.out);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                const int d0 = mt * 16 + g4;
+                if (col0) {
+                    ob[(row0 + 2 * c4) * D + d0] = o[mt][0] * inv0;
+                    ob[(row0 + 2 * c4) * D + d0 + 8] = o[mt][2] * inv0;
+                }
+                if (col1) {
+                    ob[(row0 + 2 * c4 + 1) * D + d0] = o[mt][1] * inv1;
+                    ob[(row0 + 2 * c4 + 1) * D + d0 + 8] = o[mt][3] * inv1;
+                }
+            }
+        } else {
+            // transpose the [dims x queries] fragments so a lane holds two adjacent dims of
+            // one query: 4-byte stores, one query row per 8 lanes
+            uint16_t* ob = static_cast<uint16_t*>(p.out) + (row0 + g4) * D + 2 * c4;
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                const uint32_t t0 = movmatrix_trans(cvt_bf16x2(o[mt][0] * inv0, o[mt][1] * inv1));
+                const uint32_t t1 = movmatrix_trans(cvt_bf16x2(o[mt][2] * inv0, o[mt][3] * inv1));
+                if (g4 < HP) {
+                    *reinterpret_cast<uint32_t*>(ob + mt * 16) = t0;
+                    *reinterpret_cast<uint32_t*>(ob + mt * 16 + 8) = t1;
+                }
+            }
+        }
+        if (p.lse && g4 == 0) {
+            if (col0) p.lse[row0 + 2 * c4] = (m_fin[0] + lg2(l_tot[0])) * 0.6931471805599453f;
+            if (col1) p.lse[row0 + 2 * c4 + 1] = (m_fin[1] + lg2(l_tot[1])) * 0.6931471805599453f;
+        }
+    };
+    // (o, m_fin, l_tot) -> a partial record; accumulators in fragment order: fully coalesced
+    auto store_record = [&](float* rec) {
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+            reinterpret_cast<float4*>(rec)[mt * 32 + lane] = make_float4(o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
+        if (g4 == 0) {
+            rec[D * 8 + 2 * c4] = m_fin[0];     rec[D * 8 + 2 * c4 + 1] = m_fin[1];
+            rec[D * 8 + 8 + 2 * c4] = l_tot[0]; rec[D * 8 + 8 + 2 * c4 + 1] = l_tot[1];
+        }
+    };
+    // Merge of n records in a fixed order, in one pass with running maxima: record i is the one of
+    // worker first_w + i * step (its second record if i == 0 and first_slot is set).  Record
+    // addresses do not depend on loaded data, so the unrolled loop keeps several L2 round trips in
+    // flight.  Leaves the merged (unnormalised) values in o, l_tot, m_fin.
+    auto merge_records = [&](int n, uint32_t first_w, int step, int first_slot) {
+        const float* rec0 = p.partials + (size_t)(2 * first_w) * REC;
+        const size_t rstride = (size_t)(2 * step) * REC;
+        float M[2] = {-INFINITY, -INFINITY}, Ls[2] = {0.f, 0.f};
+        float acc[MT][4];
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
+#pragma unroll 2
+        for (int i = 0; i < n; ++i) {
+            const float* r = rec0 + (size_t)i * rstride + (i == 0 ? (size_t)first_slot * REC : 0);
+            const float2 mm = __ldcg(reinterpret_cast<const float2*>(r + D * 8) + c4);
+            const float2 ll = __ldcg(reinterpret_cast<const float2*>(r + D * 8 + 8) + c4);
+            float4 x[MT];
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) x[mt] = __ldcg(reinterpret_cast<const float4*>(r) + mt * 32 + lane);
+            const float M0 = fmaxf(M[0], mm.x), M1 = fmaxf(M[1], mm.y);
+            const float a0 = ex2(M[0] - M0), a1 = ex2(M[1] - M1);      // ex2(-inf) = 0 for the first record
+            const float w0 = ex2(mm.x - M0), w1 = ex2(mm.y - M1);
+            M[0] = M0; M[1] = M1;
+            Ls[0] = fmaf(Ls[0], a0, ll.x * w0);
+            Ls[1] = fmaf(Ls[1], a1, ll.y * w1);
+#pragma unroll
+            for (int mt = 0; mt < MT; ++mt) {
+                acc[mt][0] = fmaf(acc[mt][0], a0, x[mt].x * w0);
+                acc[mt][1] = fmaf(acc[mt][1], a1, x[mt].y * w1);
+                acc[mt][2] = fmaf(acc[mt][2], a0, x[mt].z * w0);
+                acc[mt][3] = fmaf(acc[mt][3], a1, x[mt].w * w1);
+            }
+        }
+#pragma unroll
+        for (int mt = 0; mt < MT; ++mt)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) o[mt][i] = acc[mt][i];
+        l_tot[0] = Ls[0]; l_tot[1] = Ls[1];
+        m_fin[0] = M[0]; m_fin[1] = M[1];
+    };
+
     for (uint32_t tile = 0; tile < n_tiles; ++tile) {
         const int rows = min(R, cc.nv - (int)cc.t * R);
+        const bool pair_end = (cc.t + 1 == cc.nt);
+        const bool last = (tile + 1 == n_tiles);
+        // the next pair's queries are fetched while this pair's last tile is worked on
+        RowCursor cn = cc;
+        if (pair_end && !last) {
+            rcursor_next(cn, p, H, mp.groups_per_kv, R);
+            if (n_tiles - (tile + 1) < cn.nt) nxt = split_of(cn);   // the range ends inside the next pair
+            load_q(cn, qn);
+        }
 
         // ---- K tile: S^T = K . Q^T ----------------------------------------------------------
         if (!mbar_wait_bounded(bars + 8 * cslot, cphase, p.wait_limit)) { ok = false; break; }
@@ -351,162 +477,72 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
         if (cslot == 0) cphase ^= 1;
 
         // ---- end of this worker's part of the pair? -----------------------------------------
-        const bool pair_end = (cc.t + 1 == cc.nt);
-        const bool last = (tile + 1 == n_tiles);
         if (pair_end || last) {
-            float l_tot[2] = {l_run[0], l_run[1]};
+            l_tot[0] = l_run[0]; l_tot[1] = l_run[1];
 #pragma unroll
             for (int off = 4; off <= 16; off <<= 1) {
                 l_tot[0] += __shfl_xor_sync(FULL, l_tot[0], off);
                 l_tot[1] += __shfl_xor_sync(FULL, l_tot[1], off);
             }
-            float m_fin[2] = {m_run[0], m_run[1]};
+            m_fin[0] = m_run[0]; m_fin[1] = m_run[1];
 
             const bool complete = pair_end && seg_t0 == 0;
-            bool write_row = complete;
-            if (!complete) {
-                const uint64_t gs = (uint64_t)__ldg(p.pre + cc.b) * (uint64_t)H +
-                                    (uint64_t)cc.h * cc.nt;
-                const uint64_t ge = gs + cc.nt;
-                const uint32_t c_first = (uint32_t)(((gs + 1) * n_eff - 1) / total);
-                const uint32_t c_last = (uint32_t)((ge * n_eff - 1) / total);
-                const bool at_lo = (gs + seg_t0 == lo);
-                float* rec = p.partials + (size_t)(2 * w + (at_lo ? 0 : 1)) * REC;
-                // accumulators in fragment order: fully coalesced
-#pragma unroll
-                for (int mt = 0; mt < MT; ++mt)
-                    reinterpret_cast<float4*>(rec)[mt * 32 + lane] =
-                        make_float4(o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
-                if (g4 == 0) {
-                    rec[D * 8 + 2 * c4] = m_fin[0];     rec[D * 8 + 2 * c4 + 1] = m_fin[1];
-                    rec[D * 8 + 8 + 2 * c4] = l_tot[0]; rec[D * 8 + 8 + 2 * c4 + 1] = l_tot[1];
-                }
-                __threadfence();
-                __syncwarp();
-                // Merge of n records in a fixed order: record i is the one of worker
-                // first_w + i * step (its second record if i == 0 and first_slot is set).  Record
-                // addresses do not depend on loaded data, so the unrolled loops keep several L2 round
-                // trips in flight.  Leaves the merged (unnormalised) values in o, l_tot, m_fin.
-                auto merge_records = [&](int n, uint32_t first_w, int step, int first_slot) {
-                    const float* rec0 = p.partials + (size_t)(2 * first_w) * REC;
-                    const size_t rstride = (size_t)(2 * step) * REC;
-                    float M[2] = {-INFINITY, -INFINITY};
-#pragma unroll 4
-                    for (int i = 0; i < n; ++i) {
-                        const float* r = rec0 + (size_t)i * rstride + (i == 0 ? (size_t)first_slot * REC : 0);
-                        const float2 mm = __ldcg(reinterpret_cast<const float2*>(r + D * 8) + c4);
-                        M[0] = fmaxf(M[0], mm.x);
-                        M[1] = fmaxf(M[1], mm.y);
-                    }
-                    float Ls[2] = {0.f, 0.f};
-                    float acc[MT][4];
-#pragma unroll
-                    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) acc[mt][i] = 0.f;
-#pragma unroll 2
-                    for (int i = 0; i < n; ++i) {
-                        const float* r = rec0 + (size_t)i * rstride + (i == 0 ? (size_t)first_slot * REC : 0);
-                        const float2 mm = __ldcg(reinterpret_cast<const float2*>(r + D * 8) + c4);
-                        const float2 ll = __ldcg(reinterpret_cast<const float2*>(r + D * 8 + 8) + c4);
-                        const float w0 = ex2(mm.x - M[0]);
-                        const float w1 = ex2(mm.y - M[1]);
-                        Ls[0] = fmaf(ll.x, w0, Ls[0]);
-                        Ls[1] = fmaf(ll.y, w1, Ls[1]);
-#pragma unroll
-                        for (int mt = 0; mt < MT; ++mt) {
-                            const float4 x = __ldcg(reinterpret_cast<const float4*>(r) + mt * 32 + lane);
-                            acc[mt][0] = fmaf(x.x, w0, acc[mt][0]);
-                            acc[mt][1] = fmaf(x.y, w1, acc[mt][1]);
-                            acc[mt][2] = fmaf(x.z, w0, acc[mt][2]);
-                            acc[mt][3] = fmaf(x.w, w1, acc[mt][3]);
-                        }
-                    }
-#pragma unroll
-                    for (int mt = 0; mt < MT; ++mt)
-#pragma unroll
-                        for (int i = 0; i < 4; ++i) o[mt][i] = acc[mt][i];
-                    l_tot[0] = Ls[0]; l_tot[1] = Ls[1];
-                    m_fin[0] = M[0]; m_fin[1] = M[1];
-                };
-                const uint64_t lo_first = (uint64_t)c_first * total / n_eff;
-                const int first_odd = (gs != lo_first) ? 1 : 0;   // which record of c_first belongs to this pair
-                const int n_parts = (int)(c_last - c_first) + 1;
+            if (complete) {
+                write_rows(cc.b, cc.h);
+            } else {
+                const uint32_t c_first = cur.c_first;
+                const int first_odd = cur.first_odd, n_parts = cur.n_parts;
+                const bool at_lo = first_seg;
+                store_record(p.partials + (size_t)(2 * w + (at_lo ? 0 : 1)) * REC);
                 // Few parts: the contributor that arrives last merges them all.  Many parts (few
                 // pairs, long sequences): two levels - the contributors of a pair form chunks of
                 // kMmaChunk consecutive workers; the last arriver of a chunk merges the chunk's records
                 // into the record of the chunk's first worker, and the last chunk to finish merges
                 // the chunk records.  Same fixed order either way.
                 const bool two_level = n_parts > kMmaTreeMin && p.counters2 != nullptr;
-                const int k = (int)((uint32_t)w - c_first);          // this contributor's index in the pair
-                const int ck = (k / kMmaChunk) * kMmaChunk;          // its chunk's first index
-                const uint32_t cw = c_first + (uint32_t)ck;          // chunk's first worker
-                const int first_rec = (ck == 0) ? first_odd : 0;
-                const int n_chunks = (n_parts + kMmaChunk - 1) / kMmaChunk;
-                // first round: chunk level (two-level) or pair level (direct); second round: pair level
-                int32_t* tk = two_level ? p.counters2 + 2 * cw + first_rec : p.counters + c_first;
-                int n = two_level ? min(kMmaChunk, n_parts - ck) : n_parts;
-                uint32_t fw = two_level ? cw : c_first;
-                int step = 1, fslot = two_level ? first_rec : first_odd;
-                for (int round = two_level ? 0 : 1; round < 2; ++round) {
-                    int ticket = 0;
-                    if (lane == 0) ticket = atomicAdd(tk, 1);
-                    ticket = __shfl_sync(FULL, ticket, 0);
-                    if (ticket != n - 1) break;          // someone else arrives later and merges
-                    __threadfence();
-                    merge_records(n, fw, step, fslot);
-                    if (lane == 0) *tk = 0;              // ready for the next launch
-                    if (round == 1) { write_row = true; break; }
-                    // the chunk's result becomes the record of the chunk's first worker
-                    float* crec = p.partials + (size_t)(2 * cw + first_rec) * REC;
-#pragma unroll
-                    for (int mt = 0; mt < MT; ++mt)
-                        reinterpret_cast<float4*>(crec)[mt * 32 + lane] =
-                            make_float4(o[mt][0], o[mt][1], o[mt][2], o[mt][3]);
-                    if (g4 == 0) {
-                        crec[D * 8 + 2 * c4] = m_fin[0];     crec[D * 8 + 2 * c4 + 1] = m_fin[1];
-                        crec[D * 8 + 8 + 2 * c4] = l_tot[0]; crec[D * 8 + 8 + 2 * c4 + 1] = l_tot[1];
-                    }
-                    __threadfence();
-                    __syncwarp();
-                    tk = p.counters + c_first; n = n_chunks; fw = c_first; step = kMmaChunk; fslot = first_odd;
-                }
-            }
-            if (write_row) {
-                const float inv0 = 1.0f / l_tot[0], inv1 = 1.0f / l_tot[1];
-                const size_t row0 = (size_t)cc.b * mp.n_q_heads + (size_t)cc.h * HP;  // first q head
-                const bool col0 = 2 * c4 < HP, col1 = 2 * c4 + 1 < HP;
-                if (p.out_f32) {
-                    float* ob = static_cast<float*>(p.out);
-#pragma unroll
-                    for (int mt = 0; mt < MT; ++mt) {
-                        const int d0 = mt * 16 + g4;
-                        if (col0) {
-                            ob[(row0 + 2 * c4) * D + d0] = o[mt][0] * inv0;
-                            ob[(row0 + 2 * c4) * D + d0 + 8] = o[mt][2] * inv0;
-                        }
-                        if (col1) {
-                            ob[(row0 + 2 * c4 + 1) * D + d0] = o[mt][1] * inv1;
-                            ob[(row0 + 2 * c4 + 1) * D + d0 + 8] = o[mt][3] * inv1;
-                        }
+                if (!two_level) {
+                    // Post the ticket now (the release and the atomic's flight overlap with the copies
+                    // of the next tiles, already on their way); the answer is looked at after the last
+                    // tile.  Each ticket goes straight into its own variable: nothing may consume the
+                    // atomic's result here, or the warp would wait for the round trip after all.
+                    __syncwarp();   // the record's stores (all lanes) are ordered before lane 0's release
+                    if (at_lo) {
+                        if (lane == 0) pend0.ticket = atom_add_acq_rel_gpu(p.counters + c_first, 1);
+                        pend0.n = n_parts; pend0.first_odd = first_odd; pend0.b = cc.b; pend0.h = cc.h;
+                        pend0.c_first = c_first; pend0.armed = true;
+                    } else {
+                        if (lane == 0) pend1.ticket = atom_add_acq_rel_gpu(p.counters + c_first, 1);
+                        pend1.n = n_parts; pend1.first_odd = first_odd; pend1.b = cc.b; pend1.h = cc.h;
+                        pend1.c_first = c_first; pend1.armed = true;
                     }
                 } else {
-                    // transpose the [dims x queries] fragments so a lane holds two adjacent dims of
-                    // one query: 4-byte stores, one query row per 8 lanes
-                    uint16_t* ob = static_cast<uint16_t*>(p.out) + (row0 + g4) * D + 2 * c4;
-#pragma unroll
-                    for (int mt = 0; mt < MT; ++mt) {
-                        const uint32_t t0 = movmatrix_trans(cvt_bf16x2(o[mt][0] * inv0, o[mt][1] * inv1));
-                        const uint32_t t1 = movmatrix_trans(cvt_bf16x2(o[mt][2] * inv0, o[mt][3] * inv1));
-                        if (g4 < HP) {
-                            *reinterpret_cast<uint32_t*>(ob + mt * 16) = t0;
-                            *reinterpret_cast<uint32_t*>(ob + mt * 16 + 8) = t1;
-                        }
+                    __threadfence();
+                    __syncwarp();
+                    const int k = (int)((uint32_t)w - c_first);          // this contributor's index in the pair
+                    const int ck = (k / kMmaChunk) * kMmaChunk;          // its chunk's first index
+                    const uint32_t cw = c_first + (uint32_t)ck;          // chunk's first worker
+                    const int first_rec = (ck == 0) ? first_odd : 0;
+                    const int n_chunks = (n_parts + kMmaChunk - 1) / kMmaChunk;
+                    // first round: chunk level; second round: pair level
+                    int32_t* tk = p.counters2 + 2 * cw + first_rec;
+                    int n = min(kMmaChunk, n_parts - ck);
+                    uint32_t fw = cw;
+                    int step = 1, fslot = first_rec;
+                    for (int round = 0; round < 2; ++round) {
+                        int ticket = 0;
+                        if (lane == 0) ticket = atomicAdd(tk, 1);
+                        ticket = __shfl_sync(FULL, ticket, 0);
+                        if (ticket != n - 1) break;          // someone else arrives later and merges
+                        __threadfence();
+                        merge_records(n, fw, step, fslot);
+                        if (lane == 0) *tk = 0;              // ready for the next launch
+                        if (round == 1) { write_rows(cc.b, cc.h); break; }
+                        // the chunk's result becomes the record of the chunk's first worker
+                        store_record(p.partials + (size_t)(2 * cw + first_rec) * REC);
+                        __threadfence();
+                        __syncwarp();
+                        tk = p.counters + c_first; n = n_chunks; fw = c_first; step = kMmaChunk; fslot = first_odd;
                     }
-                }
-                if (p.lse && g4 == 0) {
-                    if (col0) p.lse[row0 + 2 * c4] = (m_fin[0] + lg2(l_tot[0])) * 0.6931471805599453f;
-                    if (col1) p.lse[row0 + 2 * c4 + 1] = (m_fin[1] + lg2(l_tot[1])) * 0.6931471805599453f;
                 }
             }
             m_run[0] = m_run[1] = -INFINITY;
@@ -517,8 +553,28 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
                 for (int i = 0; i < 4; ++i) o[mt][i] = 0.f;
         }
         if (!last) {
-            rcursor_next(cc, p, H, mp.groups_per_kv, R);
-            if (pair_end) { load_q(cc); seg_t0 = 0; }
+            if (pair_end) {
+                cc = cn;
+#pragma unroll
+                for (int ks = 0; ks < KS; ++ks) { qb[ks][0] = qn[ks][0]; qb[ks][1] = qn[ks][1]; }
+                seg_t0 = 0; cur = nxt; first_seg = false;
+            } else {
+                rcursor_next(cc, p, H, mp.groups_per_kv, R);
+            }
+        }
+    }
+
+    // The tickets posted above: whoever finds itself the last contributor of a pair merges it.
+    if (ok) {
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const Pending& pd = i == 0 ? pend0 : pend1;
+            if (!pd.armed) continue;
+            const int ticket = __shfl_sync(FULL, pd.ticket, 0);
+            if (ticket != pd.n - 1) continue;            // someone else arrives later and merges
+            merge_records(pd.n, pd.c_first, 1, pd.first_odd);
+            if (lane == 0) p.counters[pd.c_first] = 0;   // ready for the next launch
+            write_rows(pd.b, pd.h);
         }
     }
 

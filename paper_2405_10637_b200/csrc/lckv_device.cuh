@@ -150,6 +150,18 @@ __device__ __forceinline__ void pdl_wait_then_release()
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// Atomic add with acquire-release semantics at GPU scope, returning the old value.  Used for the
+// merge tickets: the release half publishes the partial record written before it (the record's
+// stores by the other lanes are ordered before it by the warp barrier that precedes the call), the
+// acquire half lets the arriver that finds itself last read the other contributors' records.  The
+// warp does not stall on the result until it is first used.
+__device__ __forceinline__ int32_t atom_add_acq_rel_gpu(int32_t* addr, int32_t v)
+{
+    int32_t old;
+    asm volatile("atom.acq_rel.gpu.global.add.s32 %0, [%1], %2;" : "=r"(old) : "l"(addr), "r"(v) : "memory");
+    return old;
+}
+
 __device__ __forceinline__ float ex2(float x)
 {
     float y;

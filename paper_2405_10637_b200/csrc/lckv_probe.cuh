@@ -4,6 +4,8 @@
 //   kind 0: every thread issues independent 16-byte loads (grid-stride, 8 in flight per thread) and
 //           folds them into a checksum;
 //   kind 2: the same with 32-byte loads marked evict-first in L2;
+//   (every kind can pass over the buffer several times in one launch: with a buffer that fits the L2
+//   the later passes measure the L2's read bandwidth instead of the memory's)
 //   kind 1: every warp moves 8 KB pieces into its own shared-memory ring with 1-D bulk copies, the way
 //           the attention kernels stream K and V, and reads one word of each piece.
 #pragma once
@@ -38,11 +40,13 @@ __device__ __forceinline__ uint32_t ldg_stream32_sum(const void* p)
 
 // n16 = number of 16-byte words.  sum receives the wrapped 32-bit sum of all 32-bit words read.
 __global__ void __launch_bounds__(kProbeThreads) read_stream_ldg_kernel(const uint4* __restrict__ src,
-                                                                        uint64_t n16, uint32_t* sum)
+                                                                        uint64_t n16, uint32_t* sum,
+                                                                        int repeats)
 {
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     uint32_t acc = 0;
+    for (int rep = 0; rep < repeats; ++rep) {
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     for (; i + 7 * stride < n16; i += 8 * stride) {
         uint4 v[8];
 #pragma unroll
@@ -54,6 +58,7 @@ __global__ void __launch_bounds__(kProbeThreads) read_stream_ldg_kernel(const ui
         const uint4 v = ldg_stream16(src + i);
         acc += v.x + v.y + v.z + v.w;
     }
+    }
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
     if ((threadIdx.x & 31) == 0) atomicAdd(sum, acc);
@@ -61,11 +66,13 @@ __global__ void __launch_bounds__(kProbeThreads) read_stream_ldg_kernel(const ui
 
 // The same with 32-byte loads: n32 = number of 32-byte words.
 __global__ void __launch_bounds__(kProbeThreads) read_stream_ldg32_kernel(const uint8_t* __restrict__ src,
-                                                                          uint64_t n32, uint32_t* sum)
+                                                                          uint64_t n32, uint32_t* sum,
+                                                                          int repeats)
 {
     const uint64_t stride = (uint64_t)gridDim.x * blockDim.x;
-    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     uint32_t acc = 0;
+    for (int rep = 0; rep < repeats; ++rep) {
+    uint64_t i = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
     for (; i + 3 * stride < n32; i += 4 * stride) {
         uint32_t v[4];
 #pragma unroll
@@ -73,6 +80,7 @@ __global__ void __launch_bounds__(kProbeThreads) read_stream_ldg32_kernel(const 
         acc += v[0] + v[1] + v[2] + v[3];
     }
     for (; i < n32; i += stride) acc += ldg_stream32_sum(src + i * 32);
+    }
 #pragma unroll
     for (int off = 16; off >= 1; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
     if ((threadIdx.x & 31) == 0) atomicAdd(sum, acc);
@@ -82,7 +90,8 @@ __global__ void __launch_bounds__(kProbeThreads) read_stream_ldg32_kernel(const 
 // the first word of every piece.  Waits are bounded; a wait that runs out sets *status.
 __global__ void __launch_bounds__(kProbeThreads, 1) read_stream_bulk_kernel(const uint8_t* __restrict__ src,
                                                                             uint64_t n_pieces, uint32_t* sum,
-                                                                            int32_t* status)
+                                                                            int32_t* status, int repeats,
+                                                                            float l2_keep)
 {
     extern __shared__ __align__(128) uint8_t smem[];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -96,15 +105,18 @@ __global__ void __launch_bounds__(kProbeThreads, 1) read_stream_bulk_kernel(cons
     }
     __syncwarp();
     // contiguous range per warp, like a worker's run of tiles
-    const uint64_t lo = w * n_pieces / n_warps, hi = (w + 1) * n_pieces / n_warps;
-    const uint64_t pol = make_l2_policy(0.f);
+    const uint64_t lo0 = w * n_pieces / n_warps, per = (w + 1) * n_pieces / n_warps - lo0;
+    // `repeats` passes over the warp's range, as one run of pieces: piece index i reads lo0 + i % per
+    const uint64_t lo = 0, hi = per * (uint64_t)repeats;
+    const uint64_t pol = make_l2_policy(l2_keep);
     uint64_t issued = lo;
     uint32_t islot = 0, cslot = 0, cphase = 0, acc = 0;
     bool ok = true;
     auto issue = [&]() {
         if (lane == 0) {
             mbar_expect_tx(bars + 8 * islot, kProbePiece);
-            bulk_g2s_hint(ring + islot * kProbePiece, src + issued * kProbePiece, kProbePiece, bars + 8 * islot, pol);
+            bulk_g2s_hint(ring + islot * kProbePiece, src + (lo0 + issued % per) * kProbePiece, kProbePiece,
+                          bars + 8 * islot, pol);
         }
         ++issued;
         islot = (islot + 1 == kProbeSlots) ? 0 : islot + 1;
@@ -118,7 +130,7 @@ __global__ void __launch_bounds__(kProbeThreads, 1) read_stream_bulk_kernel(cons
         cslot = (cslot + 1 == kProbeSlots) ? 0 : cslot + 1;
         if (cslot == 0) cphase ^= 1;
     }
-    if (lane == 0) atomicAdd(sum, acc);
+    if (lane == 0 && per) atomicAdd(sum, acc);
     if (!ok) {
         if (lane == 0) atomicExch(status, kStatusTimeout);
         for (int s = 0; s < kProbeSlots; ++s) {

@@ -19,14 +19,14 @@ def test_probe_checksums(nbytes):
         unit = 16 if kind == 0 else 32
         n_words = nbytes // unit * unit // 4
         acc = torch.zeros(1, dtype=torch.int32, device=dev)
-        lk.lckv_read_stream_probe(buf, nbytes, kind, acc, status)
+        lk.lckv_read_stream_probe(buf, nbytes, kind, acc, status, repeats=3)
         torch.cuda.synchronize()
-        want = int(words[:n_words].sum().item()) & 0xFFFFFFFF
+        want = 3 * int(words[:n_words].sum().item()) & 0xFFFFFFFF
         assert int(acc.item()) & 0xFFFFFFFF == want, kind
     acc = torch.zeros(1, dtype=torch.int32, device=dev)
-    lk.lckv_read_stream_probe(buf, nbytes, 1, acc, status)      # first word of every whole 8 KB piece
+    lk.lckv_read_stream_probe(buf, nbytes, 1, acc, status, repeats=2, l2_keep=0.5)   # first word of every whole 8 KB piece
     torch.cuda.synchronize()
-    want = int(words[:nbytes // 8192 * 2048:2048].sum().item()) & 0xFFFFFFFF
+    want = 2 * int(words[:nbytes // 8192 * 2048:2048].sum().item()) & 0xFFFFFFFF
     assert int(acc.item()) & 0xFFFFFFFF == want
     assert int(status.item()) == 0
 
@@ -36,8 +36,10 @@ def test_probe_rejects_bad_arguments():
     t = torch.zeros(64, dtype=torch.int32, device=dev)
     f = lk.lib().lckv_read_stream_probe
     p = t.data_ptr()
-    assert f(None, 256, 0, p, p, None) == lk.EINVAL
-    assert f(p + 4, 128, 0, p, p, None) == lk.EINVAL
-    assert f(p + 16, 128, 2, p, p, None) == lk.EINVAL
-    assert f(p, 256, 3, p, p, None) == lk.EINVAL
-    assert f(p, 8, 0, p, p, None) == lk.EINVAL
+    assert f(None, 256, 0, 1, 0.0, p, p, None) == lk.EINVAL
+    assert f(p + 4, 128, 0, 1, 0.0, p, p, None) == lk.EINVAL
+    assert f(p + 16, 128, 2, 1, 0.0, p, p, None) == lk.EINVAL
+    assert f(p, 256, 3, 1, 0.0, p, p, None) == lk.EINVAL
+    assert f(p, 8, 0, 1, 0.0, p, p, None) == lk.EINVAL
+    assert f(p, 256, 0, 0, 0.0, p, p, None) == lk.EINVAL
+    assert f(p, 256, 1, 1, 1.5, p, p, None) == lk.EINVAL
