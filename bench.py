@@ -314,8 +314,21 @@ def read_stream_probe(lk, buf, stream, nbytes=8 << 30):
         torch.cuda.synchronize()
         best = min(time_steps(f, 1, stream) for _ in range(5))
         out[name] = nbytes / (best * 1e-3) / 1e9
-    assert int(status.item()) == 0, "probe wait timed out"
     out["best"] = max(out["ldg16"], out["ldg32"], out["bulk8k"])
+    # The same kernels over a 64 MiB piece read 16 times in one launch, every line marked evict-last:
+    # the passes after the first are served by the L2 - the ceiling of a layer that re-reads a cache
+    # which the previous layer left there (TinyLlama shape at 512 tokens).
+    small, reps = min(64 << 20, nbytes), 16
+    for kind, name in ((0, "l2_ldg16"), (1, "l2_bulk8k")):
+        def g():
+            lk.lckv_read_stream_probe(buf, small, kind, acc, status, repeats=reps, l2_keep=1.0)
+        for _ in range(2):
+            g()
+        torch.cuda.synchronize()
+        best = min(time_steps(g, 1, stream) for _ in range(5))
+        out[name] = small * reps / (best * 1e-3) / 1e9
+    out["l2_resident_bytes"] = small
+    assert int(status.item()) == 0, "probe wait timed out"
     return out
 
 
@@ -489,6 +502,19 @@ def run_ours(args):
     # whole-job bytes: all ranks' units over the slowest rank's time
     value = multi.sum_over_ranks(bytes_step, dev) / (ms_step * 1e-3) / 1e9
     assert cache.lckv_cache_status() == 0, "device-side wait timed out"
+
+    # ---- optional: K further steps inside one cudaProfilerStart/Stop range (for a range-based ncu
+    #      capture, which counts DRAM bytes and L2 hits of whole steps without serialising the launches)
+    if args.profiler_range:
+        reset(B)
+        for _ in range(3):
+            step()
+        torch.cuda.synchronize()
+        torch.cuda.profiler.start()
+        for _ in range(args.profiler_range):
+            step()
+        torch.cuda.synchronize()
+        torch.cuda.profiler.stop()
 
     # ---- roofline of the dominant kernel: condensed attention launches on the shared cache ------
     n_launch = max(8, min(64, L))
@@ -786,6 +812,9 @@ def main():
                          "(default: only in the plain default run)")
     ap.add_argument("--kernel-digests", action="store_true",
                     help="print the source digests profiles/ncu_captures.json compares against, and exit")
+    ap.add_argument("--profiler-range", type=int, default=0,
+                    help="K > 0: after the timed steps, run K more steps between cudaProfilerStart and "
+                         "cudaProfilerStop (a range for ncu --replay-mode app-range)")
     ap.add_argument("--ref-rows", type=int, default=32)
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--prefill", type=int, default=0,
