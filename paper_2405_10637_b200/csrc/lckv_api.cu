@@ -89,7 +89,7 @@ struct lckv_cache {
     uint8_t* base;
     int32_t* d_lens;
     uint32_t* d_pre;
-    int32_t* d_start;
+    lckv::WorkerStart* d_start;
     int32_t* d_counters;
     int32_t* d_status;
     float* d_partials;
@@ -167,7 +167,7 @@ int mma_heads_per_pair(const lckv_config_t& c)
 
 int workers_per_sm(const lckv_config_t& c)
 {
-    return resolve_kernel_kind(c) == 2 ? lckv::kMmaWarps : lckv::kAluWarps;
+    return resolve_kernel_kind(c) == 2 ? lckv::kMmaWarps * lckv::kMmaCtas : lckv::kAluWarps * lckv::kAluCtas;
 }
 
 int partial_record_floats(const lckv_config_t& c)
@@ -224,7 +224,7 @@ void make_layout(const lckv_config_t& c, int n_slots, int n_workers, int n_kv_la
     y.off_lens = off;      off = align_up(off + (size_t)c.max_batch * 4, A);
     y.pre_stride = (int)align_up((size_t)c.max_batch + 1, 64);
     y.off_pre = off;       off = align_up(off + 2 * (size_t)y.pre_stride * 4, A);
-    y.off_start = off;     off = align_up(off + 2 * (size_t)n_workers * 4, A);
+    y.off_start = off;     off = align_up(off + 2 * (size_t)n_workers * sizeof(lckv::WorkerStart), A);
     y.off_counters = off;  off = align_up(off + 2 * 3 * (size_t)n_workers * 4, A);  // two halves of [pair tickets | chunk tickets]
     y.off_status = off;    off = align_up(off + 4, A);
     y.off_partials = off;
@@ -388,7 +388,7 @@ int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out
     p.lse = lse;
     p.lens = c->d_lens;
     p.pre = c->d_pre + (size_t)mode * c->lay.pre_stride;
-    p.start_b = c->d_start + (size_t)mode * c->n_workers;
+    p.start = c->d_start + (size_t)mode * c->n_workers;
     // consecutive launches may overlap at their edges: alternate the split-K workspace halves
     p.partials = c->d_partials + (size_t)c->ws_parity * c->partials_half_floats;
     p.counters = c->d_counters + (size_t)c->ws_parity * 3 * c->n_workers;
@@ -741,7 +741,7 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     c->n_kv_layers = 0;
     for (int l = 0; l < cfg->n_layers; ++l) c->n_kv_layers += c->plan.write_slot[l] >= 0;
     c->sm_count = sm;
-    c->grid = sm;
+    c->grid = sm * (resolve_kernel_kind(*cfg) == 2 ? lckv::kMmaCtas : lckv::kAluCtas);
     c->n_workers = sm * workers_per_sm(*cfg);
     c->kernel_kind = resolve_kernel_kind(*cfg);
     c->rows_per_tile = (c->kernel_kind == 2 ? lckv::kMmaSlotBytes : lckv::kAluSlotBytes) / (cfg->head_dim * 2);
@@ -754,7 +754,7 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     c->base = static_cast<uint8_t*>(dev_buf);
     c->d_lens = reinterpret_cast<int32_t*>(c->base + c->lay.off_lens);
     c->d_pre = reinterpret_cast<uint32_t*>(c->base + c->lay.off_pre);
-    c->d_start = reinterpret_cast<int32_t*>(c->base + c->lay.off_start);
+    c->d_start = reinterpret_cast<lckv::WorkerStart*>(c->base + c->lay.off_start);
     c->d_counters = reinterpret_cast<int32_t*>(c->base + c->lay.off_counters);
     c->d_status = reinterpret_cast<int32_t*>(c->base + c->lay.off_status);
     c->d_partials = reinterpret_cast<float*>(c->base + c->lay.off_partials);
@@ -831,7 +831,7 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
                                            lckv::kMmaSmemBytes)) &&
               cuda_ok(cudaFuncSetAttribute(lckv::project_kv_kernel,
                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                           lckv::proj_smem_bytes(256, 4))) &&
+                                           227 * 1024)) &&
               cuda_ok(cudaFuncSetAttribute(lckv::prefill_tc5_kernel<128>,
                                            cudaFuncAttributeMaxDynamicSharedMemorySize,
                                            lckv::tc5_smem_bytes<128>())) &&
@@ -1019,8 +1019,18 @@ int lckv_project_append_kv(lckv_cache_t* c, int32_t slot, const void* x, int32_t
     // batch tile = N of the MMA: any multiple of 16 up to 256; equal tiles when the batch needs several
     const int n_btiles = (batch + 255) / 256;
     const int NB = ((batch + n_btiles - 1) / n_btiles + 15) / 16 * 16;
-    int n_stages = (192 * 1024) / lckv::proj_stage_bytes(NB);
+    // k-step width: a weight row is fetched in runs of 128 * k_boxes bytes.  Runs of 256 bytes are
+    // served better by the memory than runs of 128 (fewer row activations per byte: 17.1 -> 15.2 us
+    // per call at the 7B width, B = 16); used while at least three stages still fit.
+    const int smem_budget = 222 * 1024;
+    const int k_boxes = (d_model % 128 == 0 && smem_budget / lckv::proj_stage_bytes(NB, 2) >= 3) ? 2 : 1;
+    // Stages: as many as fit beside a second CTA on the SM (so that the start of one call overlaps the
+    // tail of the kernel before it) if that leaves at least four; else as many as fit alone.
+    const int stage_bytes = lckv::proj_stage_bytes(NB, k_boxes);
+    int n_stages = (111 * 1024) / stage_bytes;
+    if (n_stages < 4) n_stages = smem_budget / stage_bytes;
     if (n_stages > 8) n_stages = 8;
+    if (n_stages < 2) return LCKV_EINVAL;
     CUtensorMap tx, tk, tv;
     if (int rc = operand_map(c, x, (uint64_t)batch, (uint64_t)d_model, NB, &tx)) return rc;
     if (int rc = operand_map(c, w_k, (uint64_t)F, (uint64_t)d_model, lckv::kProjBM, &tk)) return rc;
@@ -1048,22 +1058,26 @@ int lckv_project_append_kv(lckv_cache_t* c, int32_t slot, const void* x, int32_t
     p.rope_positions = rope_positions;
     // Few feature tiles (small batch): split d_model over a cluster so that more SMs stream weights.
     const int tiles = 2 * p.k_tiles * ((batch + NB - 1) / NB);
-    const int n_k = d_model / lckv::kProjBK;
+    const int n_k = d_model / (lckv::kProjBoxCols * k_boxes);
+    p.k_boxes = k_boxes;
     int ks = 1;
     while (ks < 8 && tiles * ks * 2 <= c->sm_count && n_k % (ks * 2) == 0 && n_k / (ks * 2) >= 4) ks *= 2;
     p.k_split = ks;
     cudaLaunchConfig_t lc = {};
     lc.gridDim = dim3(2 * p.k_tiles, (batch + NB - 1) / NB, ks);
     lc.blockDim = dim3(lckv::kProjThreads);
-    lc.dynamicSmemBytes = lckv::proj_smem_bytes(NB, n_stages);
+    lc.dynamicSmemBytes = lckv::proj_smem_bytes(NB, n_stages, k_boxes);
     lc.stream = st;
-    cudaLaunchAttribute at[1];
+    cudaLaunchAttribute at[2];
     at[0].id = cudaLaunchAttributeClusterDimension;
     at[0].val.clusterDim.x = 1;
     at[0].val.clusterDim.y = 1;
     at[0].val.clusterDim.z = ks;
+    // the kernel orders itself after its predecessor with griddepcontrol.wait (weights first)
+    at[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    at[1].val.programmaticStreamSerializationAllowed = 1;
     lc.attrs = at;
-    lc.numAttrs = 1;
+    lc.numAttrs = 2;
     if (!cuda_ok(cudaLaunchKernelEx(&lc, lckv::project_kv_kernel, p, tx, tk, tv))) return LCKV_ECUDA;
     if (advance_len) {
         if (int rc = launch_advance(c, batch, st)) return rc;
@@ -1305,7 +1319,7 @@ constexpr int kStaticMaxWorkers = LCKV_STATIC_MAX_SMS * 8;  // worker records th
 constexpr int kStaticPreStride = LCKV_STATIC_MAX_BATCH + 64;
 constexpr size_t kStOffPre = 0;
 constexpr size_t kStOffStart = kStOffPre + 2 * (size_t)kStaticPreStride * 4;
-constexpr size_t kStOffCounters = kStOffStart + 2 * (size_t)kStaticMaxWorkers * 4;
+constexpr size_t kStOffCounters = kStOffStart + 2 * (size_t)kStaticMaxWorkers * sizeof(lckv::WorkerStart);
 constexpr size_t kStOffStatus = kStOffCounters + (size_t)kStaticMaxWorkers * 4;
 constexpr size_t kStOffPartials = kStOffStatus + 256;
 constexpr size_t kStBytes = kStOffPartials + 2 * (size_t)kStaticMaxWorkers * (128 + 4) * 4;
@@ -1382,10 +1396,10 @@ extern "C" int lckv_decode_attention_static(const void* k, const void* v, const 
         base = g_static_ptr[dev].load(std::memory_order_acquire);
     }
     const int sms = g_static_sms[dev];
-    const int n_workers = sms * lckv::kAluWarps;
+    const int n_workers = sms * lckv::kAluWarps * lckv::kAluCtas;
     if (sms > LCKV_STATIC_MAX_SMS || n_workers > kStaticMaxWorkers) return LCKV_ESTATICLIMIT;
     uint32_t* d_pre = reinterpret_cast<uint32_t*>(base + kStOffPre);
-    int32_t* d_start = reinterpret_cast<int32_t*>(base + kStOffStart);
+    lckv::WorkerStart* d_start = reinterpret_cast<lckv::WorkerStart*>(base + kStOffStart);
     int32_t* d_counters = reinterpret_cast<int32_t*>(base + kStOffCounters);
     int32_t* d_status = dev_status ? dev_status : reinterpret_cast<int32_t*>(base + kStOffStatus);
 
@@ -1406,7 +1420,7 @@ extern "C" int lckv_decode_attention_static(const void* k, const void* v, const 
     p.lse = lse;
     p.lens = lens;
     p.pre = d_pre + (size_t)mode * kStaticPreStride;
-    p.start_b = d_start + (size_t)mode * n_workers;
+    p.start = d_start + (size_t)mode * n_workers;
     p.partials = reinterpret_cast<float*>(base + kStOffPartials);
     p.counters = d_counters;
     p.counters2 = nullptr;
@@ -1427,8 +1441,8 @@ extern "C" int lckv_decode_attention_static(const void* k, const void* v, const 
     const float scale = softmax_scale > 0.f ? softmax_scale : 1.0f / std::sqrt((float)head_dim);
     p.scale_log2 = scale * 1.4426950408889634f;
     if (head_dim == 128)
-        lckv::attn_alu_kernel<128><<<sms, lckv::kAluWarps * 32, lckv::kAluSmemBytes, st>>>(p);
+        lckv::attn_alu_kernel<128><<<sms * lckv::kAluCtas, lckv::kAluWarps * 32, lckv::kAluSmemBytes, st>>>(p);
     else
-        lckv::attn_alu_kernel<64><<<sms, lckv::kAluWarps * 32, lckv::kAluSmemBytes, st>>>(p);
+        lckv::attn_alu_kernel<64><<<sms * lckv::kAluCtas, lckv::kAluWarps * 32, lckv::kAluSmemBytes, st>>>(p);
     return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
 }

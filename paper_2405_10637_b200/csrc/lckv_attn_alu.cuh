@@ -17,7 +17,7 @@
 //    but looks at the answer only after its last tile, so the round trip of the atomic and the merge
 //    itself never sit between two tiles of its range.
 #pragma once
-#include "lckv_device.cuh"
+#include "lckv_small_kernels.cuh"
 
 namespace lckv {
 
@@ -34,7 +34,11 @@ namespace lckv {
 #ifndef LCKV_ALU_FFMA2
 #define LCKV_ALU_FFMA2 1
 #endif
+#ifndef LCKV_ALU_CTAS
+#define LCKV_ALU_CTAS 1
+#endif
 constexpr int kAluWarps = LCKV_ALU_WARPS;  // workers per CTA
+constexpr int kAluCtas = LCKV_ALU_CTAS;    // CTAs per SM (workers never synchronise: any split of an SM's workers into CTAs works)
 constexpr int kAluSlots = LCKV_ALU_SLOTS;  // ring slots per worker
 constexpr int kAluSlotBytes = LCKV_ALU_SLOT_BYTES;  // one tile of K or of V (a multiple of 4 KB)
 constexpr int kAluSmemBytes = kAluWarps * kAluSlots * (kAluSlotBytes + 8);
@@ -49,7 +53,7 @@ struct AttnParams {
     float* lse;               // [B, H_q] or null
     const int32_t* lens;      // [B]
     const uint32_t* pre;      // [B + 1] tile prefix for this mode
-    const int32_t* start_b;   // [n_workers] for this mode
+    const WorkerStart* start; // [n_workers] for this mode: where each worker's range begins
     float* partials;          // [2 * n_workers][D + 4]
     int32_t* counters;        // [n_workers], zero between launches
     int32_t* counters2;      // [2 * n_workers] tickets of first-level merge chunks (tensor-core kernel; may be null)
@@ -117,7 +121,7 @@ struct PageWalker {
 };
 
 template <int D, bool PAGED = false>
-__global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnParams p)
+__global__ void __launch_bounds__(kAluWarps * 32, kAluCtas) attn_alu_kernel(const AttnParams p)
 {
     constexpr int SUB = kAluSlotBytes / 4096;   // 4 KB sub-tiles per tile
     constexpr int R1 = 4096 / (D * 2);          // rows per sub-tile: 16 (D=128), 32 (D=64)
@@ -147,22 +151,13 @@ __global__ void __launch_bounds__(kAluWarps * 32, 1) attn_alu_kernel(const AttnP
 
     if (!p.early_kv) pdl_wait_then_release();
 
-    const uint64_t total = (uint64_t)__ldg(p.pre + p.B) * (uint64_t)H;
+    const WorkerStart ws = load_worker_start(p.start + w);
+    const uint64_t total = (uint64_t)__ldg(p.pre + p.B) * (uint64_t)H;   // (needed from the first cut pair on)
     const uint64_t n_eff = total < (uint64_t)p.n_workers ? total : (uint64_t)p.n_workers;
-    const bool has_work = (uint64_t)w < n_eff;
-    uint64_t lo = 0, hi = 0;
+    const uint32_t n_tiles = ws.n_tiles;
+    const bool has_work = n_tiles != 0;
     TileCursor cc;
-    cc.b = 0; cc.h = 0; cc.t = 0; cc.nt = 0; cc.nv = 0; cc.pre0 = 0;
-    if (has_work) {
-        lo = (uint64_t)w * total / n_eff;
-        hi = (uint64_t)(w + 1) * total / n_eff;
-        cc.b = __ldg(p.start_b + w);
-        cursor_load(cc, p);
-        const uint64_t rel = lo - (uint64_t)cc.pre0 * (uint64_t)H;
-        cc.h = (int32_t)(rel / cc.nt);
-        cc.t = (uint32_t)(rel % cc.nt);
-    }
-    const uint32_t n_tiles = (uint32_t)(hi - lo);
+    cc.b = ws.b; cc.h = ws.h; cc.t = ws.t; cc.nt = ws.nt; cc.nv = ws.nv; cc.pre0 = ws.pre0;
     const uint32_t n_items = 2 * n_tiles;
     TileCursor ci = cc;
 

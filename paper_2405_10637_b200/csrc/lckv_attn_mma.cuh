@@ -25,7 +25,11 @@ namespace lckv {
 #ifndef LCKV_MMA_SLOTS
 #define LCKV_MMA_SLOTS 2
 #endif
-constexpr int kMmaWarps = LCKV_MMA_WARPS;
+#ifndef LCKV_MMA_CTAS
+#define LCKV_MMA_CTAS 1
+#endif
+constexpr int kMmaWarps = LCKV_MMA_WARPS;   // workers per CTA
+constexpr int kMmaCtas = LCKV_MMA_CTAS;     // CTAs per SM
 constexpr int kMmaSlots = LCKV_MMA_SLOTS;
 #ifndef LCKV_MMA_SLOT_BYTES
 #define LCKV_MMA_SLOT_BYTES 8192
@@ -131,7 +135,7 @@ struct MmaParams {
 };
 
 template <int D, bool PAGED = false>
-__global__ void __launch_bounds__(kMmaWarps * 32, 1)
+__global__ void __launch_bounds__(kMmaWarps * 32, kMmaCtas)
 attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
                 const __grid_constant__ CUtensorMap tmV)
 {
@@ -164,23 +168,15 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
 
     if (!p.early_kv) pdl_wait_then_release();
 
-    const uint64_t total = (uint64_t)__ldg(p.pre + p.B) * (uint64_t)H;
+    const WorkerStart ws = load_worker_start(p.start + w);
+    const uint64_t total = (uint64_t)__ldg(p.pre + p.B) * (uint64_t)H;   // (needed from the first cut pair on)
     const uint64_t n_eff = total < (uint64_t)p.n_workers ? total : (uint64_t)p.n_workers;
-    const bool has_work = (uint64_t)w < n_eff;
-    uint64_t lo = 0, hi = 0;
+    const uint32_t n_tiles = ws.n_tiles;
+    const bool has_work = n_tiles != 0;
     RowCursor cc;
-    cc.b = 0; cc.h = 0; cc.t = 0; cc.nt = 0; cc.nv = 0; cc.pre0 = 0; cc.kvh = 0; cc.sub = 0; cc.row = 0;
-    if (has_work) {
-        lo = (uint64_t)w * total / n_eff;
-        hi = (uint64_t)(w + 1) * total / n_eff;
-        cc.b = __ldg(p.start_b + w);
-        rcursor_load(cc, p);
-        const uint64_t rel = lo - (uint64_t)cc.pre0 * (uint64_t)H;
-        cc.h = (int32_t)(rel / cc.nt);
-        cc.t = (uint32_t)(rel % cc.nt);
-        rcursor_seek(cc, p, mp.groups_per_kv, R);
-    }
-    const uint32_t n_tiles = (uint32_t)(hi - lo);
+    cc.b = ws.b; cc.h = ws.h; cc.t = ws.t; cc.nt = ws.nt; cc.nv = ws.nv; cc.pre0 = ws.pre0;
+    cc.kvh = 0; cc.sub = 0; cc.row = 0;
+    if (has_work) rcursor_seek(cc, p, mp.groups_per_kv, R);
     const uint32_t n_items = 2 * n_tiles;
     RowCursor ci = cc;
 

@@ -150,6 +150,10 @@ __device__ __forceinline__ void pdl_wait_then_release()
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 }
 
+// The two halves on their own, for a kernel that has work to do between them.
+__device__ __forceinline__ void pdl_release() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+
 // Atomic add with acquire-release semantics at GPU scope, returning the old value.  Used for the
 // merge tickets: the release half publishes the partial record written before it (the record's
 // stores by the other lanes are ordered before it by the warp barrier that precedes the call), the

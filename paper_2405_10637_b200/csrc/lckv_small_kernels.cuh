@@ -9,15 +9,35 @@ namespace lckv {
 // tiles: sequence b contributes ceil(n_vis[b] / R) tiles for each of its H pairs, in the order
 // (b, pair, tile), and the sequence is cut into equal contiguous ranges, one per worker warp.
 // This kernel (one block) writes, for both mask modes (n_vis = len + mode):
-//   pre[mode][b]      tiles of sequences 0..b-1 (exclusive prefix; pre[mode][B] = all tiles / H)
-//   start_b[mode][w]  the sequence in which worker w's range begins
-// so an attention worker needs two small loads to find its place.  n_vis is capped at T_cap: in
-// streaming mode (sink + recent window) a cache never holds more than T_cap rows; a negative length
-// counts as zero rows.
+//   pre[mode][b]    tiles of sequences 0..b-1 (exclusive prefix; pre[mode][B] = all tiles / H)
+//   start[mode][w]  where worker w's range begins and how long it is, with everything about that
+//                   sequence a worker needs to issue its first copy (one 32-byte load, no chain of
+//                   dependent look-ups at the start of an attention launch)
+// n_vis is capped at T_cap: in streaming mode (sink + recent window) a cache never holds more than
+// T_cap rows; a negative length counts as zero rows.
 // ---------------------------------------------------------------------------------------------
+struct __align__(32) WorkerStart {
+    int32_t b, h;        // sequence and pair in which the range begins
+    uint32_t t, nt;      // first tile within that pair; tiles per pair of sequence b
+    int32_t nv;          // visible rows of sequence b
+    uint32_t pre0;       // pre[b]
+    uint32_t n_tiles;    // length of the range (0: no work)
+    uint32_t pad;
+};
+
+__device__ __forceinline__ WorkerStart load_worker_start(const WorkerStart* p)
+{
+    const uint4 lo = __ldg(reinterpret_cast<const uint4*>(p));
+    const uint4 hi = __ldg(reinterpret_cast<const uint4*>(p) + 1);
+    WorkerStart s;
+    s.b = (int32_t)lo.x; s.h = (int32_t)lo.y; s.t = lo.z; s.nt = lo.w;
+    s.nv = (int32_t)hi.x; s.pre0 = hi.y; s.n_tiles = hi.z; s.pad = 0;
+    return s;
+}
+
 __global__ void __launch_bounds__(1024)
 plan_kernel(const int32_t* __restrict__ lens, int B, int R, int H, int n_workers,
-            uint32_t* pre, int pre_stride, int32_t* __restrict__ start_b, int T_cap)
+            uint32_t* pre, int pre_stride, WorkerStart* __restrict__ start, int T_cap)
 {
     __shared__ uint32_t warp_sums[32];
     __shared__ uint32_t carry;
@@ -58,9 +78,10 @@ plan_kernel(const int32_t* __restrict__ lens, int B, int R, int H, int n_workers
         const uint64_t total = (uint64_t)carry * (uint64_t)H;
         const uint64_t n_eff = total < (uint64_t)n_workers ? total : (uint64_t)n_workers;
         for (int w = tid; w < n_workers; w += 1024) {
-            int32_t sb = 0;
+            uint4 s0 = make_uint4(0, 0, 0, 0), s1 = s0;
             if ((uint64_t)w < n_eff) {
                 const uint64_t lo = (uint64_t)w * total / n_eff;
+                const uint64_t hi = (uint64_t)(w + 1) * total / n_eff;
                 const uint32_t x = (uint32_t)(lo / (uint64_t)H);
                 // largest b with pre[b] <= x (then pre[b+1] > x)
                 int lo_i = 0, hi_i = B;  // invariant: pre[lo_i] <= x < pre[hi_i]
@@ -68,9 +89,14 @@ plan_kernel(const int32_t* __restrict__ lens, int B, int R, int H, int n_workers
                     const int mid = (lo_i + hi_i) >> 1;
                     if (pr[mid] <= x) lo_i = mid; else hi_i = mid;
                 }
-                sb = lo_i;
+                const uint32_t pre0 = pr[lo_i], nt = pr[lo_i + 1] - pre0;
+                const uint64_t rel = lo - (uint64_t)pre0 * (uint64_t)H;
+                s0 = make_uint4((uint32_t)lo_i, (uint32_t)(rel / nt), (uint32_t)(rel % nt), nt);
+                s1 = make_uint4((uint32_t)visible_rows(lens[lo_i], mode, T_cap), pre0, (uint32_t)(hi - lo), 0u);
             }
-            start_b[mode * n_workers + w] = sb;
+            uint4* dst = reinterpret_cast<uint4*>(start + (size_t)mode * n_workers + w);
+            dst[0] = s0;
+            dst[1] = s1;
         }
         __syncthreads();
     }
