@@ -1,6 +1,7 @@
 // Host runtime and C ABI of the LCKV decode-attention library (see include/lckv.h).
 #include <cuda_runtime.h>
 
+#include <algorithm>
 #include <atomic>
 #include <cmath>
 #include <cstdio>
@@ -110,8 +111,10 @@ struct lckv_cache {
     int ws_parity;                        // which half of the split-K workspace the next launch uses
     size_t partials_half_floats;          // floats in one half of the partial records
     // CUDA graph of one step, valid for the argument pointers it was captured with
-    cudaGraphExec_t graph_exec;
-    std::vector<const void*> graph_key;
+    // Captured steps, most recently used first: a caller that alternates between a few sets of
+    // buffers (double-buffered activations) replays instead of re-capturing.
+    struct CapturedStep { std::vector<const void*> key; cudaGraphExec_t exec; };
+    std::vector<CapturedStep> graphs;
     // host-buffer step: copy streams and events (created on first use when cfg.host_staging)
     cudaStream_t s_in = nullptr, s_out = nullptr;
     std::vector<cudaEvent_t> ev;          // [0] step start, [1] k/v in, [2] all out, then per chunk in / done
@@ -524,15 +527,17 @@ int enqueue_step(lckv_cache* c, const void* const* q, void* const* out, const vo
     return launch_advance(c, batch, st);
 }
 
+constexpr size_t kMaxCapturedSteps = 4;
+
 void drop_graph(lckv_cache* c)
 {
-    if (c->graph_exec) cudaGraphExecDestroy(c->graph_exec);
-    c->graph_exec = nullptr;
-    c->graph_key.clear();
+    for (auto& g : c->graphs)
+        if (g.exec) cudaGraphExecDestroy(g.exec);
+    c->graphs.clear();
 }
 
-// One step through a CUDA graph that is re-captured whenever the argument pointers, the batch or
-// the workspace parity differ from the captured ones.
+// One step through a CUDA graph, captured the first time a set of argument pointers, batch and kept
+// L2 fraction is seen (up to kMaxCapturedSteps sets are remembered).
 int step_with_graph(lckv_cache* c, const void* const* q, void* const* out, const void* const* kn,
                     const void* const* vn, int batch, cudaStream_t st)
 {
@@ -547,8 +552,9 @@ int step_with_graph(lckv_cache* c, const void* const* q, void* const* out, const
         key.push_back(c->plan.write_slot[l] >= 0 ? kn[l] : nullptr);
         key.push_back(c->plan.write_slot[l] >= 0 ? vn[l] : nullptr);
     }
-    if (!c->graph_exec || key != c->graph_key) {
-        drop_graph(c);
+    size_t hit = 0;
+    while (hit < c->graphs.size() && c->graphs[hit].key != key) ++hit;
+    if (hit == c->graphs.size()) {
         cudaStreamCaptureStatus cs = cudaStreamCaptureStatusNone;
         if (!cuda_ok(cudaStreamIsCapturing(st, &cs))) return LCKV_ECUDA;
         // The caller is capturing already, or the stream is the legacy default stream (which
@@ -566,12 +572,19 @@ int step_with_graph(lckv_cache* c, const void* const* q, void* const* out, const
             if (g) cudaGraphDestroy(g);
             return rc ? rc : LCKV_ECUDA;
         }
-        const bool inst = cuda_ok(cudaGraphInstantiate(&c->graph_exec, g, 0));
+        cudaGraphExec_t exec = nullptr;
+        const bool inst = cuda_ok(cudaGraphInstantiate(&exec, g, 0));
         cudaGraphDestroy(g);
-        if (!inst) { c->graph_exec = nullptr; return LCKV_ECUDA; }
-        c->graph_key = key;
+        if (!inst) return LCKV_ECUDA;
+        if (c->graphs.size() >= kMaxCapturedSteps) {   // the least recently used one goes
+            cudaGraphExecDestroy(c->graphs.back().exec);
+            c->graphs.pop_back();
+        }
+        c->graphs.push_back({key, exec});
+        hit = c->graphs.size() - 1;
     }
-    if (!cuda_ok(cudaGraphLaunch(c->graph_exec, st))) return LCKV_ECUDA;
+    if (hit != 0) std::rotate(c->graphs.begin(), c->graphs.begin() + hit, c->graphs.begin() + hit + 1);
+    if (!cuda_ok(cudaGraphLaunch(c->graphs.front().exec, st))) return LCKV_ECUDA;
     c->ws_parity = c->cfg.n_layers & 1;  // where the captured step leaves it
     return LCKV_OK;
 }
@@ -788,7 +801,6 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     c->ws_parity = 0;
     c->wait_limit = lckv::kDefaultWaitLimit;
     c->partials_half_floats = 2 * (size_t)c->n_workers * partial_record_floats(*cfg);
-    c->graph_exec = nullptr;
 
     if (c->kernel_kind == 2) {
         const uint64_t rows = cfg->page_rows

@@ -348,6 +348,44 @@ def test_graph_replay_steps_match(shape):
     torch.cuda.set_stream(torch.cuda.default_stream())
 
 
+def test_graph_replay_with_alternating_buffer_sets():
+    """use_graph = 1 with a caller that rotates through several sets of buffers (more sets than the
+    library remembers captured steps for): every step, whether replayed or captured anew, matches."""
+    torch.cuda.set_stream(torch.cuda.Stream())
+    c = Case(L=4, w=2, Hq=8, Hkv=8, d=128, lens=[1, 40, 257], T_cap=300, seed=79, use_graph=1)
+    dev = c.cache.device
+    n_sets = 6
+    sets = []
+    for _ in range(n_sets):
+        q = [torch.empty((c.B, c.Hq, c.d), dtype=torch.bfloat16, device=dev) for _ in range(c.L)]
+        kn = [torch.empty((c.B, c.Hkv, c.d), dtype=torch.bfloat16, device=dev)
+              if c.plan["write_slot"][l] >= 0 else None for l in range(c.L)]
+        vn = [None if t is None else torch.empty_like(t) for t in kn]
+        outs = [torch.empty((c.B, c.Hq, c.d), dtype=torch.bfloat16, device=dev) for _ in range(c.L)]
+        sets.append((q, kn, vn, outs))
+    order = [0, 1, 0, 1, 2, 3, 4, 5, 0, 5, 1, 1]
+    for step, i in enumerate(order):
+        q, kn, vn, outs = sets[i]
+        hq, hk, hv = c.step_inputs()
+        for l in range(c.L):
+            q[l].copy_(hq[l])
+            if kn[l] is not None:
+                kn[l].copy_(hk[l]); vn[l].copy_(hv[l])
+        c.cache.lckv_layer_stack_step(q, outs, kn, vn)
+        torch.cuda.synchronize()
+        want, _ = orc.stack_step(c.L, c.w, [syn.bits(t) for t in hq],
+                                 [None if t is None else syn.bits(t) for t in hk],
+                                 [None if t is None else syn.bits(t) for t in hv],
+                                 c.hK, c.hV, c.lens, c.scale)
+        c.step_no += 1
+        for l in range(c.L):
+            compare(outs[l], want[l], f"step {step} set {i} layer {l}")
+        c.check_state()
+    c.close()
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(torch.cuda.default_stream())
+
+
 @pytest.mark.parametrize("shape", ["mha", "gqa"])
 def test_streaming_sink_and_window_cache(shape):
     """StreamingLLM-style caches (4 sinks + recent window): decode across the point where the ring

@@ -203,3 +203,31 @@ def test_prefill_on_paged_cache():
         c.check_state()
     c.step()   # and decoding continues on the same pages
     c.close()
+
+
+@pytest.mark.parametrize("n", [4096, 8192])
+def test_prefill_attention_at_the_timed_sizes(n):
+    """The shape bench.py times (7B head layout, 8 prompts of n tokens, j < i mask), checked on whole
+    query rows (all 32 heads) the oracle computes one by one: the first rows, rows around the 64- and
+    128-row tile edges, the last rows of the last query blocks, and seeded random rows."""
+    B, H, d = 8, 32, 128
+    dev = torch.device("cuda:0")
+    cfg = lk.make_config(2, 0, H, H, d, B, n)
+    cache = lk.Cache(cfg, device=dev)
+    kt, vt = cache.slot_tensors(0)
+    syn.fill_randn_bf16_(kt, 1); syn.fill_randn_bf16_(vt, 2)
+    cache.lckv_cache_reset([n] * B)
+    q = syn.randn_bf16((B, n, H, d), 3, device=dev)
+    out = cache.lckv_prefill_attention(0, lk.MODE_CONDENSED, q)
+    torch.cuda.synchronize()
+    assert cache.lckv_cache_status() == 0
+    rng = np.random.default_rng(11)
+    rows = [0, 1, 2, 63, 64, 65, 127, 128, 129, n // 2 - 1, n // 2, n - 130, n - 129, n - 128, n - 127,
+            n - 65, n - 64, n - 63, n - 2, n - 1] + [int(x) for x in rng.integers(0, n, 12)]
+    for b in (0, B - 1):
+        hk, hv = syn.bits(kt[b:b + 1]), syn.bits(vt[b:b + 1])
+        hq = syn.bits(q[b])
+        for i in rows:
+            want, _ = orc.decode_attention(hq[i:i + 1], hk, hv, np.array([i], np.int32), 0, d ** -0.5)
+            compare(out[b, i], want[0], f"seq {b} row {i}")
+    cache.close()
