@@ -503,6 +503,22 @@ def run_ours(args):
     value = multi.sum_over_ranks(bytes_step, dev) / (ms_step * 1e-3) / 1e9
     assert cache.lckv_cache_status() == 0, "device-side wait timed out"
 
+    # ---- spread of single steps (each bracketed by its own pair of events) -----------------------
+    reset(B)
+    for _ in range(3):
+        step()
+    torch.cuda.synchronize()
+    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True))
+          for _ in range(max(5, min(args.steps, 20)))]
+    for e0, e1 in ev:
+        e0.record(stream)
+        step()
+        e1.record(stream)
+    torch.cuda.synchronize()
+    us = np.array([e0.elapsed_time(e1) * 1e3 for e0, e1 in ev])
+    step_spread = {"n": len(us), "p10": float(np.percentile(us, 10)), "median": float(np.median(us)),
+                   "p90": float(np.percentile(us, 90))}
+
     # ---- optional: K further steps inside one cudaProfilerStart/Stop range (for a range-based ncu
     #      capture, which counts DRAM bytes and L2 hits of whole steps without serialising the launches)
     if args.profiler_range:
@@ -634,7 +650,7 @@ def run_ours(args):
                        "top_variant": args.top_variant, "graph": bool(args.graph),
                        "stream_sink": args.stream_sink, "page_rows": args.page_rows,
                        "cache_bytes": cache_bytes},
-            "frac_of_8TBs": value / world / NOMINAL_HBM_GBS,
+            "frac_of_8TBs": value / world / NOMINAL_HBM_GBS, "us_per_step_spread": step_spread,
             "clocks": clocks, "e2e": e2e, "gpu_launches": launches,
             "roofline": roofline, "cpu_baseline": cpu, "sweep": sweep,
             "configs": configs, "next": nxt, "clocks_extras": clocks_extras,

@@ -182,6 +182,17 @@ int lckv_cache_status(const lckv_cache_t* cache, int32_t* host_status, void* str
  */
 int lckv_cache_set_wait_limit(lckv_cache_t* cache, uint32_t polls);
 
+/*
+ * Diagnostic: lets the decode attention launches use only `workers` of the worker warps the cache was
+ * laid out for (1 ... lckv_info_t.n_workers; 0 restores all).  The tile sequence of a launch is cut
+ * into that many ranges instead, so pairs are split at other places and over other numbers of
+ * workers: running one case at several limits exercises the split-K merge (paper-side this is
+ * nothing but the log-sum-exp rule) at several split counts.  Results stay within the parity bounds
+ * at any limit; they are bitwise repeatable only at equal limits.  Takes effect from the next launch (a
+ * captured step is dropped and captured again).  EINVAL on null or a count out of range.
+ */
+int lckv_cache_set_worker_limit(lckv_cache_t* cache, int32_t workers);
+
 /* Device pointers of slot `slot`'s K and V tensors [B_max, H_kv, T_cap, d_h] bf16 (for filling
  * a cache with a prompt's keys and values, or inspecting it).  EINVAL on bad slot / null. */
 int lckv_cache_slot_ptrs(const lckv_cache_t* cache, int32_t slot, void** k, void** v);

@@ -44,6 +44,7 @@ SIGNATURES = {
     "lckv_cache_lengths": (C.c_int, [_vp, _i32p, _i32, _vp]),
     "lckv_cache_status": (C.c_int, [_vp, _i32p, _vp]),
     "lckv_cache_set_wait_limit": (C.c_int, [_vp, C.c_uint32]),
+    "lckv_cache_set_worker_limit": (C.c_int, [_vp, _i32]),
     "lckv_cache_slot_ptrs": (C.c_int, [_vp, _i32, _vpp, _vpp]),
     "lckv_cache_page_table": (C.c_int, [_vp, _i32p, _i32p]),
     "lckv_append_kv": (C.c_int, [_vp, _i32, _vp, _vp, _i32, _i32, _vp]),
@@ -209,6 +210,9 @@ class Cache:
 
     def lckv_cache_set_wait_limit(self, polls):
         _chk(lib().lckv_cache_set_wait_limit(self.h, polls), "lckv_cache_set_wait_limit")
+
+    def lckv_cache_set_worker_limit(self, workers):
+        _chk(lib().lckv_cache_set_worker_limit(self.h, workers), "lckv_cache_set_worker_limit")
 
     def lckv_cache_slot_ptrs(self, slot):
         k, v = C.c_void_p(), C.c_void_p()

@@ -87,6 +87,7 @@ struct lckv_cache {
     Layout lay;
     float scale_log2;
     int sm_count, n_workers, grid, rows_per_tile, h_pairs, kernel_kind;
+    int active_workers;                   // workers a launch uses (<= n_workers; lckv_cache_set_worker_limit)
     uint8_t* base;
     int32_t* d_lens;
     uint32_t* d_pre;
@@ -354,7 +355,7 @@ int sync_page_table(lckv_cache* c, cudaStream_t st)
 int launch_plan(lckv_cache* c, int batch, cudaStream_t st)
 {
     lckv::plan_kernel<<<1, 1024, 0, st>>>(c->d_lens, batch, c->rows_per_tile, c->h_pairs,
-                                          c->n_workers, c->d_pre, c->lay.pre_stride, c->d_start,
+                                          c->active_workers, c->d_pre, c->lay.pre_stride, c->d_start,
                                           c->cfg.max_seq);
     return cuda_ok(cudaGetLastError()) ? LCKV_OK : LCKV_ECUDA;
 }
@@ -391,7 +392,7 @@ int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out
     p.lse = lse;
     p.lens = c->d_lens;
     p.pre = c->d_pre + (size_t)mode * c->lay.pre_stride;
-    p.start = c->d_start + (size_t)mode * c->n_workers;
+    p.start = c->d_start + (size_t)mode * c->active_workers;   // (the plan kernel's stride)
     // consecutive launches may overlap at their edges: alternate the split-K workspace halves
     p.partials = c->d_partials + (size_t)c->ws_parity * c->partials_half_floats;
     p.counters = c->d_counters + (size_t)c->ws_parity * 3 * c->n_workers;
@@ -403,7 +404,7 @@ int launch_attention(lckv_cache* c, int slot, int mode, const void* q, void* out
     p.H_q = c->cfg.n_q_heads;
     p.H_kv = c->cfg.n_kv_heads;
     p.mode = mode;
-    p.n_workers = c->n_workers;
+    p.n_workers = c->active_workers;
     p.out_f32 = c->cfg.out_dtype;
     p.scale_log2 = c->scale_log2;
     p.early_kv = early ? 1 : 0;
@@ -756,6 +757,7 @@ int lckv_cache_alloc(lckv_cache_t** out, const lckv_config_t* cfg, void* dev_buf
     c->sm_count = sm;
     c->grid = sm * (resolve_kernel_kind(*cfg) == 2 ? lckv::kMmaCtas : lckv::kAluCtas);
     c->n_workers = sm * workers_per_sm(*cfg);
+    c->active_workers = c->n_workers;
     c->kernel_kind = resolve_kernel_kind(*cfg);
     c->rows_per_tile = (c->kernel_kind == 2 ? lckv::kMmaSlotBytes : lckv::kAluSlotBytes) / (cfg->head_dim * 2);
     c->h_pairs = c->kernel_kind == 2 ? cfg->n_q_heads / mma_heads_per_pair(*cfg) : cfg->n_q_heads;
@@ -950,6 +952,14 @@ int lckv_cache_set_wait_limit(lckv_cache_t* c, uint32_t polls)
     if (!c) return LCKV_EINVAL;
     c->wait_limit = polls;
     drop_graph(c);   // a captured step carries the old limit in its kernel arguments
+    return LCKV_OK;
+}
+
+int lckv_cache_set_worker_limit(lckv_cache_t* c, int32_t workers)
+{
+    if (!c || workers < 0 || workers > c->n_workers) return LCKV_EINVAL;
+    c->active_workers = workers ? workers : c->n_workers;
+    drop_graph(c);   // a captured step carries the old count in its kernel arguments
     return LCKV_OK;
 }
 

@@ -151,7 +151,10 @@ __global__ void __launch_bounds__(kAluWarps * 32, kAluCtas) attn_alu_kernel(cons
 
     if (!p.early_kv) pdl_wait_then_release();
 
-    const WorkerStart ws = load_worker_start(p.start + w);
+    // (a launch may use fewer workers than the grid holds: the others have nothing to do)
+    const bool in_range = w < p.n_workers;
+    WorkerStart ws = {0, 0, 0u, 0u, 0, 0u, 0u, 0u};
+    if (in_range) ws = load_worker_start(p.start + w);
     const uint64_t total = (uint64_t)__ldg(p.pre + p.B) * (uint64_t)H;   // (needed from the first cut pair on)
     const uint64_t n_eff = total < (uint64_t)p.n_workers ? total : (uint64_t)p.n_workers;
     const uint32_t n_tiles = ws.n_tiles;
@@ -189,7 +192,7 @@ __global__ void __launch_bounds__(kAluWarps * 32, kAluCtas) attn_alu_kernel(cons
     if (p.early_kv) pdl_wait_then_release();
 
     // Rows that see nothing (diagonal-masked first token): the zero dummy KV gives o = 0, lse = 0.
-    for (int b = w; b < p.B; b += p.n_workers) {
+    for (int b = in_range ? w : p.B; b < p.B; b += p.n_workers) {
         if (visible_rows(__ldg(p.lens + b), p.mode, p.T_cap) == 0) {
             const int esz = p.out_f32 ? 4 : 2;
             const int n16 = H * D * esz / 16;

@@ -168,7 +168,10 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
 
     if (!p.early_kv) pdl_wait_then_release();
 
-    const WorkerStart ws = load_worker_start(p.start + w);
+    // (a launch may use fewer workers than the grid holds: the others have nothing to do)
+    const bool in_range = w < p.n_workers;
+    WorkerStart ws = {0, 0, 0u, 0u, 0, 0u, 0u, 0u};
+    if (in_range) ws = load_worker_start(p.start + w);
     const uint64_t total = (uint64_t)__ldg(p.pre + p.B) * (uint64_t)H;   // (needed from the first cut pair on)
     const uint64_t n_eff = total < (uint64_t)p.n_workers ? total : (uint64_t)p.n_workers;
     const uint32_t n_tiles = ws.n_tiles;
@@ -206,7 +209,7 @@ attn_mma_kernel(const MmaParams mp, const __grid_constant__ CUtensorMap tmK,
     if (p.early_kv) pdl_wait_then_release();
 
     // Sequences that see nothing: zero rows (zero dummy KV), lse 0.
-    for (int b = w; b < p.B; b += p.n_workers) {
+    for (int b = in_range ? w : p.B; b < p.B; b += p.n_workers) {
         if (visible_rows(__ldg(p.lens + b), p.mode, p.T_cap) == 0) {
             const int esz = p.out_f32 ? 4 : 2;
             const int n16 = mp.n_q_heads * D * esz / 16;

@@ -102,3 +102,4 @@ def test_static_entry_refuses_bad_arguments_before_touching_a_gpu():
 
 def test_wait_limit_call_checks_its_handle():
     assert lk.lib().lckv_cache_set_wait_limit(None, 0) == lk.EINVAL
+    assert lk.lib().lckv_cache_set_worker_limit(None, 0) == lk.EINVAL

@@ -348,6 +348,26 @@ def test_graph_replay_steps_match(shape):
     torch.cuda.set_stream(torch.cuda.default_stream())
 
 
+@pytest.mark.parametrize("shape", ["mha", "gqa"])
+def test_same_case_at_several_split_counts(shape):
+    """The worker limit moves the cut points of a launch's tile sequence: with all workers most pairs
+    are whole or cut in two, with 37 or 5 workers the long sequences are cut differently and the short
+    ones share a worker, with 1 nothing is split at all.  Every setting must meet the oracle (the
+    split-K merge is exact up to rounding whatever the partition), also through a captured step."""
+    kw = dict(Hq=8, Hkv=8, d=128, std=1.0) if shape == "mha" else dict(Hq=16, Hkv=2, d=64, std=0.25)
+    torch.cuda.set_stream(torch.cuda.Stream())
+    c = Case(L=4, w=2, lens=[0, 1, 70, 700, 3000, 129, 64, 2047], T_cap=3100, seed=123, use_graph=1, **kw)
+    n_all = c.cache.info.n_workers
+    with pytest.raises(lk.LckvError):
+        c.cache.lckv_cache_set_worker_limit(n_all + 1)
+    for limit in (0, 37, 5, 1, n_all // 2 + 1, 0):
+        c.cache.lckv_cache_set_worker_limit(limit)
+        c.step()
+    c.close()
+    torch.cuda.synchronize()
+    torch.cuda.set_stream(torch.cuda.default_stream())
+
+
 def test_graph_replay_with_alternating_buffer_sets():
     """use_graph = 1 with a caller that rotates through several sets of buffers (more sets than the
     library remembers captured steps for): every step, whether replayed or captured anew, matches."""
